@@ -1,0 +1,153 @@
+/*
+ * grouter.h — C ABI of the B200 (sm_100a) routed SwiGLU expert layer under
+ * preemptive routing.
+ *
+ * The layer is the MoE feed-forward block of the paper's Eq. 1 (section
+ * "Mixture-of-Experts"),   y = sum_i r(x)_i f_i(x),   evaluated with the
+ * coefficient vector r(x) *loaded* instead of computed: a frozen router ran
+ * ahead of time and cached, per token, k expert ids and k gate scores (section
+ * "Decoupling Preemptive Routing"; appendix "Efficiency Experiment Detail",
+ * Pre-Dispatch: uint8 ids, bfloat16 scores).  f_i is a bias-free SwiGLU FFN,
+ *   f_i(x) = W_d[i] ( silu(W_g[i] x) * (W_u[i] x) ).
+ *
+ * Conventions for every call
+ *   - All tensor arguments are DEVICE pointers unless the name ends in _host.
+ *     They are caller-owned, contiguous, row-major and 16-byte aligned.
+ *   - bf16 tensors are passed as `const void*` / `void*`.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work and return; they do not synchronise, and after
+ *     grouter_create they do not allocate.
+ *   - Return value: GROUTER_OK (0) or a negative GROUTER_ERR_* for problems the
+ *     host can see.  Problems only the device can see (an expert id out of
+ *     range, a bounded wait that ran out) set a sticky status word; the
+ *     kernels keep every access in bounds and finish, and grouter_status()
+ *     reports it.  Nothing traps.
+ *   - Outputs are overwritten, never accumulated into.
+ *
+ * Sizes: T tokens, d model width, ffn expert hidden width, k experts per token,
+ * E_src ids that may appear in idx, E_tgt experts that own weights
+ * (E_tgt == E_src unless a fold map is given), R = T*k routed slots,
+ * slot s = t*k + j.  Required: d % 8 == 0, ffn % 8 == 0, 1 <= E_tgt <= 1024,
+ * R < 2^31 - 2^18.
+ */
+#ifndef GROUTER_H_
+#define GROUTER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  GROUTER_OK = 0,
+  GROUTER_ERR_INVALID_ARG = -1,   /* NULL pointer, non-positive size, bad enum         */
+  GROUTER_ERR_MISALIGNED = -2,    /* a tensor pointer is not 16-byte aligned           */
+  GROUTER_ERR_UNSUPPORTED = -3,   /* d or ffn not a multiple of 8, E_tgt > 1024, ...   */
+  GROUTER_ERR_INVALID_STATE = -4, /* fwd/bwd before plan, bwd before fwd               */
+  GROUTER_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed                 */
+  GROUTER_ERR_BAD_INDEX = -6,     /* device saw an expert id or fold target out of range */
+  GROUTER_ERR_TIMEOUT = -7,       /* a bounded device-side wait ran out                */
+  GROUTER_ERR_NO_DEVICE = -8      /* no usable CUDA device / not sm_100                */
+};
+
+enum { GROUTER_IDX_U8 = 0, GROUTER_IDX_I32 = 1 };
+enum { GROUTER_GATE_BF16 = 0, GROUTER_GATE_F32 = 1 };
+
+typedef struct grouter_ctx grouter_ctx; /* opaque */
+
+typedef struct {
+  int32_t T, d, ffn, E_src, E_tgt, k;
+  int32_t idx_dtype;  /* GROUTER_IDX_U8 (the paper's cache format, E_src <= 256) or GROUTER_IDX_I32 */
+  int32_t gate_dtype; /* GROUTER_GATE_BF16 (the paper's cache format) or GROUTER_GATE_F32           */
+  int32_t flags;      /* reserved, pass 0 */
+} grouter_dims;
+
+/* Creates a context for one layer shape on the current CUDA device.  Host call;
+ * the only call that allocates: a few MB of device memory for the padded copy
+ * of the plan, the tile list, per-block histograms and the status word.
+ * Errors: INVALID_ARG, UNSUPPORTED, NO_DEVICE, CUDA. */
+int grouter_create(grouter_ctx** out, const grouter_dims* dims);
+void grouter_destroy(grouter_ctx* ctx);
+
+/* Bytes of device workspace grouter_moe_fwd / grouter_moe_bwd need for `dims`.
+ * The workspace carries the expert-ordered activations from fwd to the
+ * matching bwd (gathered tokens, gate/up pre-activations, gated hidden state),
+ * so it must not be touched in between.  Rows are padded per expert to a
+ * multiple of 128, so it is sized for T*k + 128*E_tgt rows.  0 on bad dims. */
+size_t grouter_workspace_bytes(const grouter_dims* dims);
+/* Extra bytes grouter_moe_step_host needs after the workspace proper. */
+size_t grouter_host_staging_bytes(const grouter_dims* dims);
+
+/* Routing-plan build: a stable counting sort of the R slots by target expert.
+ *   e_s            = fold_map ? fold_map[idx[s]] : idx[s]
+ *   counts[e]      = #{ s : e_s == e }
+ *   offsets[e]     = sum_{e' < e} counts[e'],   offsets[E_tgt] = R
+ *   slot_to_row[s] = offsets[e_s] + #{ s' < s : e_s' == e_s }
+ *   row_to_slot    = inverse permutation
+ * The fold map is the compact form of the paper's binary folding matrix M
+ * (section "Expert Folding", Matrix Folding): fold_map[i] = the j with M_ij = 1.
+ * It is applied to the cached ids after top-k, so a token may own several rows
+ * of one target expert.
+ *   idx         [T,k] uint8 or int32 (dims.idx_dtype), values in [0,E_src)
+ *   fold_map    [E_src] int32 in [0,E_tgt), or NULL for the identity
+ *   counts      [E_tgt] int32 out          offsets     [E_tgt+1] int32 out
+ *   row_to_slot [R] int32 out              slot_to_row [R] int32 out
+ * The context keeps a 128-row-padded copy of the plan for fwd/bwd; one plan
+ * may serve any number of fwd/bwd calls (all MoE layers of a micro-batch share
+ * the same frozen router; section "Decoupled Structure Extraction").
+ * An id outside [0,E_src) or a fold target outside [0,E_tgt) is treated as
+ * expert 0 and sets the sticky status GROUTER_ERR_BAD_INDEX. */
+int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+                 int32_t* row_to_slot, int32_t* slot_to_row, void* stream);
+
+/* Forward, Eq. 1:  Y[t,:] = sum_j gates[t,j] * f_{e(t,j)}(X[t,:]).
+ *   X     [T,d] bf16             gates [T,k] bf16 or f32 (dims.gate_dtype), used as given
+ *   W_gu  [E_tgt, 2*ffn, d] bf16: rows 0..ffn-1 gate projection, ffn..2ffn-1 up projection
+ *   W_d   [E_tgt, d, ffn] bf16   Y     [T,d] bf16 out (fp32 accumulate)
+ *   workspace: grouter_workspace_bytes(dims) bytes
+ * Needs a prior grouter_plan on the same ctx (else INVALID_STATE). */
+int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const void* W_gu, const void* W_d, void* Y,
+                    void* workspace, void* stream);
+
+/* Backward of grouter_moe_fwd for L with dL/dY = dY (expert gradient as in the
+ * paper's appendix on joint optimisation: dL/dtheta_e = dL/dy * sum_i r_i * grad f_i).
+ *   dY     [T,d] bf16                 dX     [T,d] bf16 out
+ *   dW_gu  [E_tgt, 2*ffn, d] f32 out  dW_d   [E_tgt, d, ffn] f32 out
+ *   dgates [T,k] f32 out: dgates[t,j] = <dY[t,:], f_{e(t,j)}(X[t,:])> (gates are leaf inputs)
+ * Experts that received no slot get exact zeros in dW_*.  Uses the workspace
+ * contents left by the matching grouter_moe_fwd (else INVALID_STATE). */
+int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void* gates, const void* W_gu,
+                    const void* W_d, void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace,
+                    void* stream);
+
+/* One whole step from HOST buffers: copies idx, gates, X, dY to the device
+ * (cudaMemcpyAsync on `stream`; pass pinned memory for real overlap), runs plan,
+ * fwd and bwd, and copies Y, dX, dgates back.  Weights, weight gradients and
+ * fold_map stay on the device.  `workspace` must hold
+ * grouter_workspace_bytes + grouter_host_staging_bytes.  Returns after
+ * enqueueing; synchronise the stream before reading the host outputs. */
+int grouter_moe_step_host(grouter_ctx* ctx, const void* idx_host, const void* gates_host, const void* X_host,
+                          const void* dY_host, const int32_t* fold_map, const void* W_gu, const void* W_d,
+                          void* Y_host, void* dX_host, float* dgates_host, float* dW_gu, float* dW_d,
+                          void* workspace, void* stream);
+
+/* Synchronises `stream` and returns the sticky device status (GROUTER_OK,
+ * GROUTER_ERR_BAD_INDEX, GROUTER_ERR_TIMEOUT) or GROUTER_ERR_CUDA; clears it. */
+int grouter_status(grouter_ctx* ctx, void* stream);
+
+const char* grouter_strerror(int code);
+
+/* Component check of the tensor-core core used by every grouped GEMM (no
+ * counterpart in the paper): C[M,N] (f32) = A * B with bf16 operands.
+ *   a_mn_major == 0: A stored [M,K] (K contiguous); != 0: A stored [K,M].
+ *   b_mn_major == 0: B stored [N,K] (K contiguous); != 0: B stored [K,N].
+ * M, N, K multiples of 8.  `status` is a device int32 the kernel ORs error bits into. */
+int grouter_dense_gemm(const void* A, int a_mn_major, const void* B, int b_mn_major, float* C, int32_t M, int32_t N,
+                       int32_t K, int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GROUTER_H_ */

@@ -1,0 +1,183 @@
+"""ctypes binding of libgrouter.so (the C ABI in include/grouter.h).
+
+Argument marshalling only: every step of the layer runs in the CUDA library.
+torch is used for device memory and streams.  There is no fallback: if the
+library cannot be loaded this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+IDX_U8, IDX_I32 = 0, 1
+GATE_BF16, GATE_F32 = 0, 1
+
+EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
+           "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
+           "grouter_dense_gemm"]
+
+
+class GrouterDims(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("T", "d", "ffn", "E_src", "E_tgt", "k", "idx_dtype", "gate_dtype", "flags")]
+
+
+class GrouterError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads (building in-tree first if stale or absent) and types the library."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.LIB
+        if not os.path.exists(path) or os.environ.get("GROUTER_REBUILD"):
+            _build.build()
+    lib = ctypes.CDLL(path)
+    vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+    lib.grouter_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(GrouterDims)]
+    lib.grouter_create.restype = ctypes.c_int
+    lib.grouter_destroy.argtypes = [vp]
+    lib.grouter_destroy.restype = None
+    lib.grouter_workspace_bytes.argtypes = [ctypes.POINTER(GrouterDims)]
+    lib.grouter_workspace_bytes.restype = ctypes.c_size_t
+    lib.grouter_host_staging_bytes.argtypes = [ctypes.POINTER(GrouterDims)]
+    lib.grouter_host_staging_bytes.restype = ctypes.c_size_t
+    lib.grouter_plan.argtypes = [vp, vp, i32p, i32p, i32p, i32p, i32p, vp]
+    lib.grouter_plan.restype = ctypes.c_int
+    lib.grouter_moe_fwd.argtypes = [vp] * 8
+    lib.grouter_moe_fwd.restype = ctypes.c_int
+    lib.grouter_moe_bwd.argtypes = [vp] * 12
+    lib.grouter_moe_bwd.restype = ctypes.c_int
+    lib.grouter_moe_step_host.argtypes = [vp] * 15
+    lib.grouter_moe_step_host.restype = ctypes.c_int
+    lib.grouter_status.argtypes = [vp, vp]
+    lib.grouter_status.restype = ctypes.c_int
+    lib.grouter_strerror.argtypes = [ctypes.c_int]
+    lib.grouter_strerror.restype = ctypes.c_char_p
+    lib.grouter_dense_gemm.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, f32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
+    lib.grouter_dense_gemm.restype = ctypes.c_int
+    if path == _build.LIB:
+        _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().grouter_strerror(code).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise GrouterError(code, what)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class GrouterLayer:
+    """One layer shape: owns the context and the workspace; thin calls into the C ABI."""
+
+    def __init__(self, T: int, d: int, ffn: int, E_src: int, k: int, E_tgt: Optional[int] = None, idx_dtype: int = IDX_U8,
+                 gate_dtype: int = GATE_BF16, device: str = "cuda:0", host_staging: bool = False):
+        self.lib = load_library()
+        self.device = torch.device(device)
+        self.dims = GrouterDims(T, d, ffn, E_src, E_src if E_tgt is None else E_tgt, k, idx_dtype, gate_dtype, 0)
+        self.T, self.d, self.ffn, self.k = T, d, ffn, k
+        self.E_src, self.E_tgt = E_src, self.dims.E_tgt
+        self.R = T * k
+        with torch.cuda.device(self.device):
+            h = ctypes.c_void_p()
+            _check(self.lib.grouter_create(ctypes.byref(h), ctypes.byref(self.dims)), "grouter_create")
+            self.ctx = h
+            n = self.lib.grouter_workspace_bytes(ctypes.byref(self.dims))
+            if n == 0:
+                raise GrouterError(-3, "grouter_workspace_bytes")
+            self.workspace_bytes = n
+            if host_staging:
+                n += self.lib.grouter_host_staging_bytes(ctypes.byref(self.dims))
+            self.workspace = torch.empty(n, dtype=torch.uint8, device=self.device)
+        i32 = dict(dtype=torch.int32, device=self.device)
+        self.counts = torch.empty(self.E_tgt, **i32)
+        self.offsets = torch.empty(self.E_tgt + 1, **i32)
+        self.row_to_slot = torch.empty(self.R, **i32)
+        self.slot_to_row = torch.empty(self.R, **i32)
+
+    def close(self) -> None:
+        if getattr(self, "ctx", None):
+            self.lib.grouter_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def plan(self, idx: torch.Tensor, fold_map: Optional[torch.Tensor] = None):
+        """idx [T,k] uint8/int32 (device); fold_map [E_src] int32 or None.  Results land in
+        self.counts / offsets / row_to_slot / slot_to_row."""
+        _check(self.lib.grouter_plan(self.ctx, _ptr(idx), _ptr(fold_map), _ptr(self.counts), _ptr(self.offsets),
+                                     _ptr(self.row_to_slot), _ptr(self.slot_to_row), _stream()), "grouter_plan")
+        return self.counts, self.offsets, self.row_to_slot, self.slot_to_row
+
+    def forward(self, X, gates, W_gu, W_d, Y=None):
+        if Y is None:
+            Y = torch.empty_like(X)
+        _check(self.lib.grouter_moe_fwd(self.ctx, _ptr(X), _ptr(gates), _ptr(W_gu), _ptr(W_d), _ptr(Y), _ptr(self.workspace),
+                                        _stream()), "grouter_moe_fwd")
+        return Y
+
+    def backward(self, dY, X, gates, W_gu, W_d, dX=None, dW_gu=None, dW_d=None, dgates=None):
+        f32 = dict(dtype=torch.float32, device=self.device)
+        dX = torch.empty_like(X) if dX is None else dX
+        dW_gu = torch.empty(W_gu.shape, **f32) if dW_gu is None else dW_gu
+        dW_d = torch.empty(W_d.shape, **f32) if dW_d is None else dW_d
+        dgates = torch.empty((self.T, self.k), **f32) if dgates is None else dgates
+        _check(self.lib.grouter_moe_bwd(self.ctx, _ptr(dY), _ptr(X), _ptr(gates), _ptr(W_gu), _ptr(W_d), _ptr(dX), _ptr(dW_gu),
+                                        _ptr(dW_d), _ptr(dgates), _ptr(self.workspace), _stream()), "grouter_moe_bwd")
+        return dX, dW_gu, dW_d, dgates
+
+    def step_host(self, idx_h, gates_h, X_h, dY_h, fold_map, W_gu, W_d, Y_h, dX_h, dgates_h, dW_gu, dW_d):
+        """Whole step from pinned host tensors (idx, gates, X, dY in; Y, dX, dgates out)."""
+        _check(self.lib.grouter_moe_step_host(self.ctx, _ptr(idx_h), _ptr(gates_h), _ptr(X_h), _ptr(dY_h), _ptr(fold_map), _ptr(W_gu),
+                                              _ptr(W_d), _ptr(Y_h), _ptr(dX_h), _ptr(dgates_h), _ptr(dW_gu), _ptr(dW_d),
+                                              _ptr(self.workspace), _stream()), "grouter_moe_step_host")
+
+    def status(self) -> int:
+        """Synchronises the current stream; returns 0 or a negative GROUTER_ERR_* device status."""
+        return self.lib.grouter_status(self.ctx, _stream())
+
+    def check_status(self) -> None:
+        _check(self.status(), "device status")
+
+
+def dense_gemm(A: torch.Tensor, a_mn_major: bool, B: torch.Tensor, b_mn_major: bool, M: int, N: int, K: int) -> torch.Tensor:
+    """C[M,N] f32 = A*B on the tcgen05 core (component check).  A is [M,K] or, MN-major, [K,M]; B is [N,K] or [K,N]."""
+    lib = load_library()
+    C = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    status = torch.zeros(1, dtype=torch.int32, device=A.device)
+    _check(lib.grouter_dense_gemm(_ptr(A), int(a_mn_major), _ptr(B), int(b_mn_major), _ptr(C), M, N, K, _ptr(status), _stream()),
+           "grouter_dense_gemm")
+    torch.cuda.synchronize(A.device)
+    if int(status.item()) != 0:
+        raise GrouterError(-7, "grouter_dense_gemm device status")
+    return C

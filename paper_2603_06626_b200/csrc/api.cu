@@ -1,0 +1,271 @@
+// C-ABI entry points: argument checks, context, workspace carve-up and the
+// launch sequence of the forward and backward passes.
+#include <new>
+
+#include "common.cuh"
+
+using namespace grouter;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_dims(const grouter_dims* dm) {
+  if (!dm) return GROUTER_ERR_INVALID_ARG;
+  if (dm->T < 1 || dm->d < 1 || dm->ffn < 1 || dm->E_src < 1 || dm->E_tgt < 1 || dm->k < 1) return GROUTER_ERR_INVALID_ARG;
+  if (dm->idx_dtype != GROUTER_IDX_U8 && dm->idx_dtype != GROUTER_IDX_I32) return GROUTER_ERR_INVALID_ARG;
+  if (dm->gate_dtype != GROUTER_GATE_BF16 && dm->gate_dtype != GROUTER_GATE_F32) return GROUTER_ERR_INVALID_ARG;
+  if (dm->d % 8 || dm->ffn % 8) return GROUTER_ERR_UNSUPPORTED;
+  if (dm->E_tgt > 1024 || dm->k > 32) return GROUTER_ERR_UNSUPPORTED;
+  if (dm->idx_dtype == GROUTER_IDX_U8 && dm->E_src > 256) return GROUTER_ERR_UNSUPPORTED;
+  const int64_t R = (int64_t)dm->T * dm->k;
+  if (R >= (int64_t)2147483647 - (1 << 18)) return GROUTER_ERR_UNSUPPORTED;
+  return GROUTER_OK;
+}
+
+inline int64_t r_pad_max(const grouter_dims& dm) {
+  const int64_t R = (int64_t)dm.T * dm.k;
+  return (R + ROW_TILE - 1) / ROW_TILE * ROW_TILE + (int64_t)ROW_TILE * dm.E_tgt;
+}
+
+struct Staging {  // device copies of the per-step host inputs/outputs of grouter_moe_step_host
+  size_t idx, gates, X, dY, Y, dX, dgates, counts, offsets, r2s, s2r, bytes;
+};
+Staging staging_layout(const grouter_dims& dm) {
+  Staging s{};
+  const size_t R = (size_t)dm.T * dm.k, Td = (size_t)dm.T * dm.d;
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
+  s.idx = take(R * (dm.idx_dtype == GROUTER_IDX_U8 ? 1 : 4));
+  s.gates = take(R * (dm.gate_dtype == GROUTER_GATE_BF16 ? 2 : 4));
+  s.X = take(Td * 2);
+  s.dY = take(Td * 2);
+  s.Y = take(Td * 2);
+  s.dX = take(Td * 2);
+  s.dgates = take(R * 4);
+  s.counts = take((size_t)dm.E_tgt * 4);
+  s.offsets = take((size_t)(dm.E_tgt + 1) * 4);
+  s.r2s = take(R * 4);
+  s.s2r = take(R * 4);
+  s.bytes = off;
+  return s;
+}
+
+}  // namespace
+
+namespace grouter {
+Workspace carve_workspace(const grouter_dims& dm, int64_t Rp, void* base) {
+  Workspace w{};
+  char* b = static_cast<char*>(base);
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
+  const size_t rd = (size_t)Rp * dm.d * 2, rf = (size_t)Rp * dm.ffn * 2;
+  const size_t oXp = take(rd), oG = take(rf), oU = take(rf), oH = take(rf), oO = take(rd), odY = take(rd), odGU = take(2 * rf);
+  const size_t oPart = take((size_t)((dm.ffn + 255) / 256) * Rp * 4);
+  w.bytes = off;
+  if (b) {
+    w.Xp = reinterpret_cast<__nv_bfloat16*>(b + oXp);
+    w.G = reinterpret_cast<__nv_bfloat16*>(b + oG);
+    w.U = reinterpret_cast<__nv_bfloat16*>(b + oU);
+    w.Hs = reinterpret_cast<__nv_bfloat16*>(b + oH);
+    w.O = reinterpret_cast<__nv_bfloat16*>(b + oO);
+    w.dYp = reinterpret_cast<__nv_bfloat16*>(b + odY);
+    w.dGU = reinterpret_cast<__nv_bfloat16*>(b + odGU);
+    w.dgate_part = reinterpret_cast<float*>(b + oPart);
+  }
+  return w;
+}
+}  // namespace grouter
+
+extern "C" {
+
+const char* grouter_strerror(int code) {
+  switch (code) {
+    case GROUTER_OK: return "ok";
+    case GROUTER_ERR_INVALID_ARG: return "invalid argument";
+    case GROUTER_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case GROUTER_ERR_UNSUPPORTED: return "unsupported size or type";
+    case GROUTER_ERR_INVALID_STATE: return "call order: plan before fwd, fwd before bwd";
+    case GROUTER_ERR_CUDA: return "CUDA call failed";
+    case GROUTER_ERR_BAD_INDEX: return "expert id or fold target out of range (seen on device)";
+    case GROUTER_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case GROUTER_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+    default: return "unknown error";
+  }
+}
+
+size_t grouter_workspace_bytes(const grouter_dims* dims) {
+  if (check_dims(dims) != GROUTER_OK) return 0;
+  return carve_workspace(*dims, r_pad_max(*dims), nullptr).bytes;
+}
+
+size_t grouter_host_staging_bytes(const grouter_dims* dims) {
+  if (check_dims(dims) != GROUTER_OK) return 0;
+  return staging_layout(*dims).bytes;
+}
+
+int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
+  if (!out) return GROUTER_ERR_INVALID_ARG;
+  *out = nullptr;
+  const int rc = check_dims(dims);
+  if (rc != GROUTER_OK) return rc;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return GROUTER_ERR_NO_DEVICE;
+  int major = 0, sms = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GROUTER_ERR_NO_DEVICE;
+  if (major != 10) return GROUTER_ERR_NO_DEVICE;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  grouter_ctx* c = new (std::nothrow) grouter_ctx();
+  if (!c) return GROUTER_ERR_INVALID_ARG;
+  c->dims = *dims;
+  c->device = dev;
+  c->num_sms = sms;
+  c->R = (int64_t)dims->T * dims->k;
+  c->R_pad_max = r_pad_max(*dims);
+  c->max_m_tiles = (int)(c->R_pad_max / ROW_TILE);
+  c->geom = plan_geom(c->R);
+  c->planned = c->forwarded = false;
+  const int E = dims->E_tgt;
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
+  const size_t o_pad = take((size_t)(E + 1) * 4), o_shift = take((size_t)E * 4), o_pb = take((size_t)E * 4);
+  const size_t o_te = take((size_t)c->max_m_tiles * 4), o_nt = take(4), o_s2p = take((size_t)c->R * 4);
+  const size_t o_p2s = take((size_t)c->R_pad_max * 4), o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
+  if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
+    delete c;
+    return GROUTER_ERR_CUDA;
+  }
+  if (cudaMemset(c->d_block, 0, off) != cudaSuccess) {
+    cudaFree(c->d_block);
+    delete c;
+    return GROUTER_ERR_CUDA;
+  }
+  char* b = static_cast<char*>(c->d_block);
+  c->pp.pad_offsets = reinterpret_cast<int32_t*>(b + o_pad);
+  c->pp.row_shift = reinterpret_cast<int32_t*>(b + o_shift);
+  c->pp.pad_begin = reinterpret_cast<int32_t*>(b + o_pb);
+  c->pp.tile_expert = reinterpret_cast<int32_t*>(b + o_te);
+  c->pp.n_m_tiles = reinterpret_cast<int32_t*>(b + o_nt);
+  c->pp.slot_to_prow = reinterpret_cast<int32_t*>(b + o_s2p);
+  c->pp.prow_to_slot = reinterpret_cast<int32_t*>(b + o_p2s);
+  c->pp.blk_prefix = reinterpret_cast<int32_t*>(b + o_bp);
+  c->pp.ticket = reinterpret_cast<unsigned int*>(b + o_tk);
+  c->pp.status = reinterpret_cast<int32_t*>(b + o_st);
+  *out = c;
+  return GROUTER_OK;
+}
+
+void grouter_destroy(grouter_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->d_block) cudaFree(ctx->d_block);
+  delete ctx;
+}
+
+int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+                 int32_t* row_to_slot, int32_t* slot_to_row, void* stream) {
+  if (!ctx || !idx || !counts || !offsets || !row_to_slot || !slot_to_row) return GROUTER_ERR_INVALID_ARG;
+  if (!aligned16(idx) || !aligned16(counts) || !aligned16(offsets) || !aligned16(row_to_slot) || !aligned16(slot_to_row) ||
+      (fold_map && !aligned16(fold_map)))
+    return GROUTER_ERR_MISALIGNED;
+  if (!fold_map && ctx->dims.E_src != ctx->dims.E_tgt) return GROUTER_ERR_INVALID_ARG;
+  if (launch_plan(ctx, idx, fold_map, counts, offsets, row_to_slot, slot_to_row, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return GROUTER_ERR_CUDA;
+  ctx->planned = true;
+  ctx->forwarded = false;
+  return GROUTER_OK;
+}
+
+int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const void* W_gu, const void* W_d, void* Y,
+                    void* workspace, void* stream) {
+  if (!ctx || !X || !gates || !W_gu || !W_d || !Y || !workspace) return GROUTER_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(gates) || !aligned16(W_gu) || !aligned16(W_d) || !aligned16(Y) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return GROUTER_ERR_MISALIGNED;
+  if (!ctx->planned) return GROUTER_ERR_INVALID_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Workspace ws = carve_workspace(ctx->dims, ctx->R_pad_max, workspace);
+  if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(X), ws.Xp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_grouped_gemm(ctx, MODE_UP, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_grouped_gemm(ctx, MODE_DOWN, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  ctx->forwarded = true;
+  return GROUTER_OK;
+}
+
+int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void* gates, const void* W_gu, const void* W_d,
+                    void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace, void* stream) {
+  if (!ctx || !dY || !X || !gates || !W_gu || !W_d || !dX || !dW_gu || !dW_d || !dgates || !workspace) return GROUTER_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(gates) || !aligned16(W_gu) || !aligned16(W_d) || !aligned16(dX) ||
+      !aligned16(dW_gu) || !aligned16(dW_d) || !aligned16(dgates) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return GROUTER_ERR_MISALIGNED;
+  if (!ctx->planned || !ctx->forwarded) return GROUTER_ERR_INVALID_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Workspace ws = carve_workspace(ctx->dims, ctx->R_pad_max, workspace);
+  const int n_part = (ctx->dims.ffn + 255) / 256;
+  if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(dY), ws.dYp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_grouped_gemm(ctx, MODE_DH, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_grouped_gemm(ctx, MODE_WGRAD_D, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_grouped_gemm(ctx, MODE_DX, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_grouped_gemm(ctx, MODE_WGRAD_GU, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(dX), ws.dgate_part, n_part, dgates, st) != cudaSuccess)
+    return GROUTER_ERR_CUDA;
+  return GROUTER_OK;
+}
+
+int grouter_moe_step_host(grouter_ctx* ctx, const void* idx_host, const void* gates_host, const void* X_host, const void* dY_host,
+                          const int32_t* fold_map, const void* W_gu, const void* W_d, void* Y_host, void* dX_host,
+                          float* dgates_host, float* dW_gu, float* dW_d, void* workspace, void* stream) {
+  if (!ctx || !idx_host || !gates_host || !X_host || !dY_host || !Y_host || !dX_host || !dgates_host || !workspace)
+    return GROUTER_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return GROUTER_ERR_MISALIGNED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const grouter_dims& dm = ctx->dims;
+  const size_t ws_bytes = carve_workspace(dm, ctx->R_pad_max, nullptr).bytes;
+  const Staging sg = staging_layout(dm);
+  char* sb = static_cast<char*>(workspace) + ws_bytes;
+  const size_t R = (size_t)dm.T * dm.k, Td = (size_t)dm.T * dm.d;
+  const size_t idx_b = R * (dm.idx_dtype == GROUTER_IDX_U8 ? 1 : 4), gate_b = R * (dm.gate_dtype == GROUTER_GATE_BF16 ? 2 : 4);
+  if (cudaMemcpyAsync(sb + sg.idx, idx_host, idx_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemcpyAsync(sb + sg.gates, gates_host, gate_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemcpyAsync(sb + sg.X, X_host, Td * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemcpyAsync(sb + sg.dY, dY_host, Td * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  int rc = grouter_plan(ctx, sb + sg.idx, fold_map, reinterpret_cast<int32_t*>(sb + sg.counts), reinterpret_cast<int32_t*>(sb + sg.offsets),
+                        reinterpret_cast<int32_t*>(sb + sg.r2s), reinterpret_cast<int32_t*>(sb + sg.s2r), stream);
+  if (rc != GROUTER_OK) return rc;
+  rc = grouter_moe_fwd(ctx, sb + sg.X, sb + sg.gates, W_gu, W_d, sb + sg.Y, workspace, stream);
+  if (rc != GROUTER_OK) return rc;
+  rc = grouter_moe_bwd(ctx, sb + sg.dY, sb + sg.X, sb + sg.gates, W_gu, W_d, sb + sg.dX, dW_gu, dW_d,
+                       reinterpret_cast<float*>(sb + sg.dgates), workspace, stream);
+  if (rc != GROUTER_OK) return rc;
+  if (cudaMemcpyAsync(Y_host, sb + sg.Y, Td * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemcpyAsync(dX_host, sb + sg.dX, Td * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemcpyAsync(dgates_host, sb + sg.dgates, R * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  return GROUTER_OK;
+}
+
+int grouter_status(grouter_ctx* ctx, void* stream) {
+  if (!ctx) return GROUTER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t h = 0;
+  if (cudaMemcpyAsync(&h, ctx->pp.status, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (h != 0) {
+    if (cudaMemsetAsync(ctx->pp.status, 0, 4, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    if (h & STATUS_TIMEOUT) return GROUTER_ERR_TIMEOUT;
+    return GROUTER_ERR_BAD_INDEX;
+  }
+  return GROUTER_OK;
+}
+
+int grouter_dense_gemm(const void* A, int a_mn_major, const void* B, int b_mn_major, float* C, int32_t M, int32_t N, int32_t K,
+                       int32_t* status, void* stream) {
+  if (!A || !B || !C || !status || M < 1 || N < 1 || K < 1) return GROUTER_ERR_INVALID_ARG;
+  if (M % 8 || N % 8 || K % 8) return GROUTER_ERR_UNSUPPORTED;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(C)) return GROUTER_ERR_MISALIGNED;
+  if (launch_dense_gemm(A, a_mn_major, B, b_mn_major, C, M, N, K, status, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return GROUTER_ERR_CUDA;
+  return GROUTER_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,102 @@
+// Shared declarations of the CUDA path (host launchers, context, status bits).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "grouter.h"
+
+namespace grouter {
+
+// Sticky device status bits (ORed into ctx->d_status).
+constexpr int STATUS_BAD_INDEX = 1;
+constexpr int STATUS_TIMEOUT = 2;
+
+constexpr int ROW_TILE = 128;        // rows of one GEMM tile; expert segments are padded to it
+constexpr int PLAN_THREADS = 256;    // 8 warps per plan block
+constexpr int PLAN_WARPS = PLAN_THREADS / 32;
+constexpr int PLAN_MIN_CHUNK = 2048; // slots per plan block (lower bound)
+constexpr int PLAN_MAX_BLOCKS = 1184;// 148 SMs x 8 resident blocks
+
+struct PlanGeom {
+  int chunk;    // slots per block, multiple of 256
+  int nblk;     // blocks
+};
+
+inline PlanGeom plan_geom(int64_t R) {
+  int64_t chunk = (R + PLAN_MAX_BLOCKS - 1) / PLAN_MAX_BLOCKS;
+  if (chunk < PLAN_MIN_CHUNK) chunk = PLAN_MIN_CHUNK;
+  chunk = (chunk + PLAN_THREADS - 1) / PLAN_THREADS * PLAN_THREADS;
+  PlanGeom g;
+  g.chunk = (int)chunk;
+  g.nblk = (int)((R + chunk - 1) / chunk);
+  if (g.nblk < 1) g.nblk = 1;
+  return g;
+}
+
+// Device-side copy of the plan in the 128-row-padded layout the GEMMs use.
+struct PaddedPlan {
+  int32_t* pad_offsets;   // [E_tgt+1] first padded row of each expert; [E_tgt] = rows in use
+  int32_t* row_shift;     // [E_tgt]   pad_offsets[e] - offsets[e]
+  int32_t* pad_begin;     // [E_tgt]   first pad row of expert e (pad_offsets[e] + counts[e])
+  int32_t* tile_expert;   // [max_m_tiles] expert of each 128-row tile
+  int32_t* n_m_tiles;     // [1]
+  int32_t* slot_to_prow;  // [R]
+  int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows
+  int32_t* blk_prefix;    // [E_tgt * nblk] per-block histogram, then exclusive prefix over blocks
+  unsigned int* ticket;   // [1] last-block-done counter
+  int32_t* status;        // [1] sticky status bits
+};
+
+}  // namespace grouter
+
+struct grouter_ctx {
+  grouter_dims dims;
+  int device;
+  int64_t R;
+  int64_t R_pad_max;      // round_up(R,128) + 128*E_tgt
+  int max_m_tiles;
+  grouter::PlanGeom geom;
+  grouter::PaddedPlan pp;
+  void* d_block;          // one allocation backing pp
+  bool planned;
+  bool forwarded;
+  int num_sms;
+};
+
+namespace grouter {
+
+// Workspace carve-up (all offsets 256-byte aligned).
+struct Workspace {
+  __nv_bfloat16* Xp;    // [R_pad_max, d]   gathered tokens
+  __nv_bfloat16* G;     // [R_pad_max, F]   gate pre-activation
+  __nv_bfloat16* U;     // [R_pad_max, F]   up pre-activation
+  __nv_bfloat16* Hs;    // [R_pad_max, F]   gate-scaled hidden state g*silu(G)*U
+  __nv_bfloat16* O;     // [R_pad_max, d]   expert outputs (fwd) / dXp (bwd)
+  __nv_bfloat16* dYp;   // [R_pad_max, d]   gathered upstream gradient
+  __nv_bfloat16* dGU;   // [R_pad_max, 2F]  [dG | dU]
+  float* dgate_part;    // [ceil(F/256), R_pad_max] partial row sums for d-gate
+  size_t bytes;
+};
+Workspace carve_workspace(const grouter_dims& dm, int64_t R_pad_max, void* base);
+
+// ---- launchers (each returns a cudaError_t from the launch) ----
+cudaError_t launch_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+                        int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st);
+
+// dst[prow,:] = src[slot/k,:] for every routed slot; pad rows zero-filled.
+cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st);
+// out[t,:] = sum_j src[slot_to_prow[t*k+j],:] (fp32 sum in slot order); optionally
+// dgates[t,j] = sum_n dgate_part[n][prow].
+cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part,
+                               int n_part, float* dgates, cudaStream_t st);
+
+enum GemmMode { MODE_UP = 0, MODE_DOWN = 1, MODE_DH = 2, MODE_DX = 3, MODE_WGRAD_D = 4, MODE_WGRAD_GU = 5, MODE_DENSE = 6 };
+
+cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace& ws, const void* gates, const void* W_gu,
+                                const void* W_d, float* dW_gu, float* dW_d, cudaStream_t st);
+cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,
+                              cudaStream_t st);
+
+}  // namespace grouter

@@ -1,0 +1,143 @@
+// HBM-bound row movers between token order and expert-contiguous (padded) order.
+//
+// Both run token-major with one warp per token and 128-bit accesses, so each
+// token row is read (scatter) or written (reduce) exactly once and every
+// routed row is touched exactly once: (T + R) * d * 2 bytes, the algorithmic
+// minimum.
+//   scatter_rows: dst[slot_to_prow[t*k+j], :] = src[t, :]      (gather of X / dY)
+//   reduce_rows : out[t, :] = sum_j src[slot_to_prow[t*k+j], :]  (Eq. 1 combine; dX)
+// The gate weights are already folded into the rows by the GEMM epilogues, so
+// the combine is an unweighted fp32 sum in slot order (deterministic).
+#include "common.cuh"
+
+namespace grouter {
+
+constexpr int MOVE_THREADS = 256;
+constexpr int MOVE_WARPS = MOVE_THREADS / 32;
+
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_v4(void* p, const uint4& v) {
+  asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+__global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
+                                                                    const int32_t* __restrict__ slot_to_prow,
+                                                                    const int32_t* __restrict__ pad_begin,
+                                                                    const int32_t* __restrict__ pad_offsets, int T, int k, int d, int E) {
+  const int lane = threadIdx.x & 31;
+  const int gwarp = blockIdx.x * MOVE_WARPS + (threadIdx.x >> 5);
+  const int nwarps = gridDim.x * MOVE_WARPS;
+  const int units = d >> 3;  // 16-byte units per row
+  for (int t = gwarp; t < T; t += nwarps) {
+    const int my_prow = lane < k ? __ldg(slot_to_prow + (size_t)t * k + lane) : 0;
+    const char* s = reinterpret_cast<const char*>(src + (size_t)t * d);
+    for (int u0 = 0; u0 < units; u0 += 128) {
+      uint4 v[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int u = u0 + i * 32 + lane;
+        if (u < units) v[i] = ld_nc_v4(s + (size_t)u * 16);
+      }
+      for (int j = 0; j < k; ++j) {
+        const int prow = __shfl_sync(0xffffffffu, my_prow, j);
+        char* o = reinterpret_cast<char*>(dst + (size_t)prow * d);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int u = u0 + i * 32 + lane;
+          if (u < units) st_v4(o + (size_t)u * 16, v[i]);
+        }
+      }
+    }
+  }
+  // zero the pad rows of every expert segment
+  const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+  for (int e = gwarp; e < E; e += nwarps) {
+    const int r0 = pad_begin[e], r1 = pad_offsets[e + 1];
+    for (int r = r0; r < r1; ++r) {
+      char* o = reinterpret_cast<char*>(dst + (size_t)r * d);
+      for (int u = lane; u < units; u += 32) st_v4(o + (size_t)u * 16, z);
+    }
+  }
+}
+
+__device__ __forceinline__ void acc_bf16x8(float (&a)[8], const uint4& v) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(p[i]);
+    a[2 * i] += f.x;
+    a[2 * i + 1] += f.y;
+  }
+}
+
+__global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ out,
+                                                                   const int32_t* __restrict__ slot_to_prow, int T, int k, int d,
+                                                                   const float* __restrict__ dgate_part, int n_part, size_t part_stride,
+                                                                   float* __restrict__ dgates) {
+  const int lane = threadIdx.x & 31;
+  const int gwarp = blockIdx.x * MOVE_WARPS + (threadIdx.x >> 5);
+  const int nwarps = gridDim.x * MOVE_WARPS;
+  const int units = d >> 3;
+  for (int t = gwarp; t < T; t += nwarps) {
+    const int my_prow = lane < k ? __ldg(slot_to_prow + (size_t)t * k + lane) : 0;
+    if (dgates != nullptr && lane < k) {
+      float g = 0.f;
+      for (int n = 0; n < n_part; ++n) g += dgate_part[(size_t)n * part_stride + my_prow];
+      dgates[(size_t)t * k + lane] = g;
+    }
+    char* o = reinterpret_cast<char*>(out + (size_t)t * d);
+    for (int u0 = 0; u0 < units; u0 += 64) {
+      float a0[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      float a1[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      const int ua = u0 + lane, ub = u0 + 32 + lane;
+#pragma unroll 4
+      for (int j = 0; j < k; ++j) {
+        const int prow = __shfl_sync(0xffffffffu, my_prow, j);
+        const char* s = reinterpret_cast<const char*>(src + (size_t)prow * d);
+        if (ua < units) acc_bf16x8(a0, ld_nc_v4(s + (size_t)ua * 16));
+        if (ub < units) acc_bf16x8(a1, ld_nc_v4(s + (size_t)ub * 16));
+      }
+      if (ua < units) {
+        uint4 v;
+        __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(a0[2 * i], a0[2 * i + 1]);
+        st_v4(o + (size_t)ua * 16, v);
+      }
+      if (ub < units) {
+        uint4 v;
+        __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(a1[2 * i], a1[2 * i + 1]);
+        st_v4(o + (size_t)ub * 16, v);
+      }
+    }
+  }
+}
+
+static int mover_grid(const grouter_ctx* ctx, int T) {
+  const int want = (T + MOVE_WARPS - 1) / MOVE_WARPS;
+  const int cap = ctx->num_sms * 8;
+  return want < cap ? (want < 1 ? 1 : want) : cap;
+}
+
+cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st) {
+  const grouter_dims& dm = ctx->dims;
+  scatter_rows_kernel<<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_prow, ctx->pp.pad_begin,
+                                                                      ctx->pp.pad_offsets, dm.T, dm.k, dm.d, dm.E_tgt);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part, int n_part,
+                               float* dgates, cudaStream_t st) {
+  const grouter_dims& dm = ctx->dims;
+  reduce_rows_kernel<<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_prow, dm.T, dm.k, dm.d, dgate_part, n_part,
+                                                                     (size_t)ctx->R_pad_max, dgates);
+  return cudaGetLastError();
+}
+
+}  // namespace grouter

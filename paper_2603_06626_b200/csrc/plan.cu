@@ -1,0 +1,241 @@
+// Routing-plan build: a stable counting sort of the R = T*k slots by target
+// expert, in two launches.
+//
+//   plan_hist_kernel    every block histograms a contiguous chunk of slots
+//                       (one private histogram per warp, built with
+//                       __match_any_sync so no atomics are needed); the last
+//                       block to finish turns the per-block histograms into
+//                       exclusive prefixes over blocks, scans the expert
+//                       counts into offsets, and lays out the 128-row-padded
+//                       segments and the tile list the grouped GEMMs walk.
+//   plan_permute_kernel every warp walks its sub-chunk in slot order; the rank
+//                       of a slot among equal experts is (block prefix) +
+//                       (earlier warps of the block) + (earlier lanes), which
+//                       makes the permutation stable and bit-reproducible.
+//
+// The fold map is the compact form of the paper's binary folding matrix M
+// (section "Expert Folding"): e_s = fold_map[idx_s].
+#include "common.cuh"
+
+namespace grouter {
+
+template <typename IdxT>
+__device__ __forceinline__ int load_expert(const IdxT* __restrict__ idx, int s, const int32_t* __restrict__ fold_map, int E_src,
+                                           int E_tgt, int32_t* status) {
+  int raw = (int)idx[s];
+  bool bad = false;
+  if ((unsigned)raw >= (unsigned)E_src) {
+    bad = true;
+    raw = 0;
+  }
+  int e = fold_map ? __ldg(fold_map + raw) : raw;
+  if ((unsigned)e >= (unsigned)E_tgt) {
+    bad = true;
+    e = 0;
+  }
+  if (bad) atomicOr(status, STATUS_BAD_INDEX);
+  return e;
+}
+
+// Per-warp histograms of this block's chunk into hist[w*E + e] (smem, pre-zeroed).
+template <typename IdxT>
+__device__ __forceinline__ void warp_histogram(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map, int R, int E_src,
+                                               int E_tgt, int chunk, int32_t* hist, int32_t* status) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wlen = chunk / PLAN_WARPS;
+  const int base = blockIdx.x * chunk + warp * wlen;
+  int32_t* h = hist + warp * E_tgt;
+  for (int i = 0; i < wlen; i += 32) {
+    const int s = base + i + lane;
+    const bool valid = s < R;
+    const int e = valid ? load_expert(idx, s, fold_map, E_src, E_tgt, status) : -1;
+    const unsigned mask = __match_any_sync(0xffffffffu, e);
+    if (valid && lane == __ffs(mask) - 1) h[e] += __popc(mask);
+    __syncwarp();
+    if (base + i + 32 >= R) break;
+  }
+}
+
+template <typename IdxT>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                 int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
+                                                                 int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+  extern __shared__ int32_t sm[];  // max(PLAN_WARPS*E, 3*E+3) ints
+  __shared__ int s_last;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
+  __syncthreads();
+  warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, pp.status);
+  __syncthreads();
+  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+    int tot = 0;
+#pragma unroll
+    for (int w = 0; w < PLAN_WARPS; ++w) tot += sm[w * E_tgt + e];
+    pp.blk_prefix[e * nblk + blockIdx.x] = tot;
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned t = atomicAdd(pp.ticket, 1u);
+    s_last = (t == (unsigned)(nblk - 1));
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // ---- last block: prefixes over blocks, offsets, padded layout, tile list ----
+  int32_t* s_cnt = sm;                    // [E]
+  int32_t* s_off = sm + E_tgt;            // [E+1]
+  int32_t* s_pad = sm + 2 * E_tgt + 1;    // [E+1]
+  __syncthreads();
+  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
+    int carry = 0;
+    for (int b0 = 0; b0 < nblk; b0 += 32) {
+      const int b = b0 + lane;
+      const int v = b < nblk ? __ldcg(pp.blk_prefix + e * nblk + b) : 0;
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (b < nblk) pp.blk_prefix[e * nblk + b] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_cnt[e] = carry;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int per = (E_tgt + 31) / 32;
+    const int e0 = min(lane * per, E_tgt), e1 = min(e0 + per, E_tgt);
+    int sum = 0, psum = 0;
+    for (int e = e0; e < e1; ++e) {
+      sum += s_cnt[e];
+      psum += (s_cnt[e] + ROW_TILE - 1) / ROW_TILE * ROW_TILE;
+    }
+    int isum = sum, ipsum = psum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int a = __shfl_up_sync(0xffffffffu, isum, o);
+      const int b = __shfl_up_sync(0xffffffffu, ipsum, o);
+      if (lane >= o) {
+        isum += a;
+        ipsum += b;
+      }
+    }
+    int off = isum - sum, poff = ipsum - psum;
+    for (int e = e0; e < e1; ++e) {
+      s_off[e] = off;
+      s_pad[e] = poff;
+      off += s_cnt[e];
+      poff += (s_cnt[e] + ROW_TILE - 1) / ROW_TILE * ROW_TILE;
+    }
+    if (lane == 31) {
+      s_off[E_tgt] = isum;
+      s_pad[E_tgt] = ipsum;
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e <= E_tgt; e += PLAN_THREADS) {
+    offsets[e] = s_off[e];
+    pp.pad_offsets[e] = s_pad[e];
+    if (e < E_tgt) {
+      counts[e] = s_cnt[e];
+      pp.row_shift[e] = s_pad[e] - s_off[e];
+      pp.pad_begin[e] = s_pad[e] + s_cnt[e];
+    }
+  }
+  const int n_tiles = s_pad[E_tgt] / ROW_TILE;
+  if (tid == 0) {
+    *pp.n_m_tiles = n_tiles;
+    *pp.ticket = 0u;  // ready for the next plan
+  }
+  // expert of every 128-row tile: the last e with pad_offsets[e] <= first row of the tile
+  for (int t = tid; t < n_tiles; t += PLAN_THREADS) {
+    const int row = t * ROW_TILE;
+    int lo = 0, hi = E_tgt;  // invariant: s_pad[lo] <= row < s_pad[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_pad[mid] <= row) lo = mid; else hi = mid;
+    }
+    pp.tile_expert[t] = lo;
+  }
+  // pad rows carry no slot
+  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
+    const int r0 = s_pad[e] + s_cnt[e], r1 = s_pad[e + 1];
+    for (int r = r0 + lane; r < r1; r += 32) pp.prow_to_slot[r] = -1;
+  }
+}
+
+template <typename IdxT>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_permute_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                    int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
+                                                                    const int32_t* __restrict__ offsets, int32_t* __restrict__ row_to_slot,
+                                                                    int32_t* __restrict__ slot_to_row) {
+  extern __shared__ int32_t sm[];  // PLAN_WARPS*E + E ints
+  int32_t* s_shift = sm + PLAN_WARPS * E_tgt;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
+  __syncthreads();
+  warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, pp.status);
+  __syncthreads();
+  // per-warp histogram -> first row of (block, warp, expert)
+  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+    int base = offsets[e] + pp.blk_prefix[e * nblk + blockIdx.x];
+#pragma unroll
+    for (int w = 0; w < PLAN_WARPS; ++w) {
+      const int t = sm[w * E_tgt + e];
+      sm[w * E_tgt + e] = base;
+      base += t;
+    }
+    s_shift[e] = pp.row_shift[e];
+  }
+  __syncthreads();
+  const int wlen = chunk / PLAN_WARPS;
+  const int base = blockIdx.x * chunk + warp * wlen;
+  int32_t* cur = sm + warp * E_tgt;
+  const unsigned lt = (1u << lane) - 1u;
+  for (int i = 0; i < wlen; i += 32) {
+    const int s = base + i + lane;
+    const bool valid = s < R;
+    const int e = valid ? load_expert(idx, s, fold_map, E_src, E_tgt, pp.status) : -1;
+    const unsigned mask = __match_any_sync(0xffffffffu, e);
+    const int row = valid ? cur[e] + __popc(mask & lt) : 0;
+    __syncwarp();
+    if (valid && lane == 31 - __clz(mask)) cur[e] = row + 1;
+    __syncwarp();
+    if (valid) {
+      const int prow = row + s_shift[e];
+      slot_to_row[s] = row;
+      row_to_slot[row] = s;
+      pp.slot_to_prow[s] = prow;
+      pp.prow_to_slot[prow] = s;
+    }
+    if (base + i + 32 >= R) break;
+  }
+}
+
+template <typename IdxT>
+static cudaError_t launch_plan_t(grouter_ctx* ctx, const IdxT* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+                                 int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
+  const grouter_dims& dm = ctx->dims;
+  const int R = (int)ctx->R, E = dm.E_tgt;
+  const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
+  const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 3 * E + 3) ? PLAN_WARPS * E : 3 * E + 3);
+  const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
+  plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  plan_permute_kernel<IdxT><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, offsets, row_to_slot,
+                                                             slot_to_row);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+                        int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
+  if (ctx->dims.idx_dtype == GROUTER_IDX_U8)
+    return launch_plan_t<uint8_t>(ctx, (const uint8_t*)idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st);
+  return launch_plan_t<int32_t>(ctx, (const int32_t*)idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st);
+}
+
+}  // namespace grouter

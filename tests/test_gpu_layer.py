@@ -1,0 +1,200 @@
+"""Forward/backward parity of the CUDA path against the fp64 oracle.
+
+Bar: relative Frobenius error <= 1e-2 per tensor (bf16 storage, fp32 accumulate
+against an unrounded fp64 oracle); experts without slots must give exact zeros.
+Small workloads are compared in full; the large ones on sampled tokens (Y, dX,
+dgates) and sampled experts (dW_gu, dW_d), each compared element by element.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import grouter_oracle as orc
+from paper_2603_06626_b200 import synth
+from tests.gpu_util import bits_to_bf16, to_dev
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-2
+
+
+def run_gpu(w, li, gate_f32=False, idx_i32=False):
+    """One plan + fwd + bwd through the C ABI.  Returns device tensors."""
+    from paper_2603_06626_b200 import binding
+    layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt,
+                                 idx_dtype=binding.IDX_I32 if idx_i32 else binding.IDX_U8,
+                                 gate_dtype=binding.GATE_F32 if gate_f32 else binding.GATE_BF16)
+    idx = to_dev(li.idx.astype(np.int32) if idx_i32 else li.idx)
+    fm = None if li.fold_map is None else to_dev(li.fold_map)
+    gates = bits_to_bf16(li.gates)
+    if gate_f32:
+        gates = gates.float()
+    X, dY = bits_to_bf16(li.X), bits_to_bf16(li.dY)
+    W_gu, W_d = bits_to_bf16(li.W_gu), bits_to_bf16(li.W_d)
+    layer.plan(idx, fm)
+    Y = layer.forward(X, gates, W_gu, W_d)
+    dX, dW_gu, dW_d, dgates = layer.backward(dY, X, gates, W_gu, W_d)
+    layer.check_status()
+    out = dict(Y=Y, dX=dX, dW_gu=dW_gu, dW_d=dW_d, dgates=dgates, counts=layer.counts.cpu().numpy())
+    layer.close()
+    return out
+
+
+def oracle_inputs(li):
+    w = li.w
+    X = synth.bf16_bits_to_f64(li.X)
+    dY = synth.bf16_bits_to_f64(li.dY)
+    gates = synth.bf16_bits_to_f64(li.gates)
+    if li.W_gu is not None:
+        weights = orc.Weights(getter=lambda e: (synth.bf16_bits_to_f64(li.W_gu[e]), synth.bf16_bits_to_f64(li.W_d[e])), ffn=w.ffn)
+    else:
+        weights = orc.Weights(getter=lambda e: (synth.bf16_bits_to_f64(synth.expert_W_gu(w, e)),
+                                                synth.bf16_bits_to_f64(synth.expert_W_d(w, e))), ffn=w.ffn)
+    return X, dY, gates, weights
+
+
+def f64(t):
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def check_full(w, li, out):
+    X, dY, gates, weights = oracle_inputs(li)
+    Y = orc.moe_forward(X, li.idx, gates, weights, w.E_tgt, li.fold_map)
+    dX, dgates, dW = orc.moe_backward(dY, X, li.idx, gates, weights, w.E_tgt, li.fold_map)
+    errs = {"Y": orc.rel_frobenius(f64(out["Y"]), Y), "dX": orc.rel_frobenius(f64(out["dX"]), dX),
+            "dgates": orc.rel_frobenius(f64(out["dgates"]), dgates)}
+    dWgu = np.stack([dW[e][0] for e in range(w.E_tgt)])
+    dWd = np.stack([dW[e][1] for e in range(w.E_tgt)])
+    errs["dW_gu"] = orc.rel_frobenius(f64(out["dW_gu"]), dWgu)
+    errs["dW_d"] = orc.rel_frobenius(f64(out["dW_d"]), dWd)
+    for e in range(w.E_tgt):
+        if out["counts"][e] == 0:
+            assert not out["dW_gu"][e].any() and not out["dW_d"][e].any(), f"expert {e} has no slot: dW must be exact zeros"
+        else:
+            assert orc.rel_frobenius(f64(out["dW_gu"][e]), dW[e][0]) < TOL, f"dW_gu[{e}]"
+            assert orc.rel_frobenius(f64(out["dW_d"][e]), dW[e][1]) < TOL, f"dW_d[{e}]"
+    for t in out.values():
+        if torch.is_tensor(t):
+            assert torch.isfinite(t).all()
+    assert max(errs.values()) < TOL, errs
+    return errs
+
+
+def check_sampled(w, li, out, n_tokens, experts):
+    X, dY, gates, weights = oracle_inputs(li)
+    rng = np.random.default_rng(1234 + w.seed)
+    tokens = np.sort(rng.choice(w.T, size=min(n_tokens, w.T), replace=False))
+    Y = orc.moe_forward(X, li.idx, gates, weights, w.E_tgt, li.fold_map, tokens=tokens)
+    dX, dgates = orc.moe_backward_tokens(dY, X, li.idx, gates, weights, w.E_tgt, li.fold_map, tokens=tokens)
+    tk = torch.from_numpy(tokens).to(out["Y"].device)
+    errs = {"Y": orc.rel_frobenius(f64(out["Y"][tk]), Y), "dX": orc.rel_frobenius(f64(out["dX"][tk]), dX),
+            "dgates": orc.rel_frobenius(f64(out["dgates"][tk]), dgates)}
+    for e in experts:
+        dWgu, dWd = orc.moe_backward_expert(dY, X, li.idx, gates, weights, w.E_tgt, int(e), li.fold_map)
+        if out["counts"][e] == 0:
+            assert not dWgu.any() and not dWd.any()
+            assert not out["dW_gu"][e].any() and not out["dW_d"][e].any()
+        else:
+            errs[f"dW_gu[{e}]"] = orc.rel_frobenius(f64(out["dW_gu"][e]), dWgu)
+            errs[f"dW_d[{e}]"] = orc.rel_frobenius(f64(out["dW_d"][e]), dWd)
+    for name in ("Y", "dX", "dgates", "dW_gu", "dW_d"):
+        assert torch.isfinite(out[name]).all(), name
+    assert max(errs.values()) < TOL, errs
+    return errs
+
+
+def pick_experts(counts, n_random, seed):
+    """heaviest, lightest non-empty, every empty one, and a few random ones"""
+    nz = np.nonzero(counts)[0]
+    chosen = {int(nz[np.argmax(counts[nz])]), int(nz[np.argmin(counts[nz])])}
+    chosen |= {int(e) for e in np.nonzero(counts == 0)[0]}
+    rng = np.random.default_rng(seed)
+    chosen |= {int(e) for e in rng.choice(len(counts), size=min(n_random, len(counts)), replace=False)}
+    return sorted(chosen)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_full_parity(name):
+    w = synth.WORKLOADS[name]
+    li = synth.make_layer_inputs(w)
+    out = run_gpu(w, li)
+    errs = check_full(w, li, out)
+    print(name, errs)
+
+
+def test_fine_fold_sampled():
+    w = synth.WORKLOADS["fine_fold"]
+    li = synth.make_layer_inputs(w)
+    out = run_gpu(w, li)
+    assert out["counts"].sum() == w.R
+    print(check_sampled(w, li, out, 512, pick_experts(out["counts"], 1, 0)[:3]))
+
+
+def test_skewed_sampled_with_empty_experts():
+    w = synth.WORKLOADS["skewed"]
+    li = synth.make_layer_inputs(w)
+    out = run_gpu(w, li)
+    assert (out["counts"] == 0).sum() == 4
+    print(check_sampled(w, li, out, 512, pick_experts(out["counts"], 1, 1)))
+
+
+def test_large_sampled():
+    w = synth.WORKLOADS["large"]
+    li = synth.make_layer_inputs(w)
+    out = run_gpu(w, li)
+    counts = out["counts"]
+    nz = np.nonzero(counts)[0]
+    light = int(nz[np.argmin(counts[nz])])
+    median = int(nz[np.argsort(counts[nz])[len(nz) // 2]])
+    heavy = int(nz[np.argmax(counts[nz])])
+    print(check_sampled(w, li, out, 256, [light, median, heavy]))
+
+
+@pytest.mark.parametrize("T,d,F,E,k,kw", [
+    (300, 64, 64, 1, 1, {}),                       # dense special case, one ragged tile
+    (257, 128, 72, 5, 3, {}),                      # F not a multiple of 64; segments far below one tile
+    (1000, 720, 720, 32, 4, {}),                   # a model shape from the paper's configuration table
+    (640, 384, 344, 128, 8, {}),                   # another: more experts than tiles per expert
+    (900, 512, 704, 64, 6, {"load": "zipf", "zipf_s": 1.3, "n_dead": 7}),
+    (512, 1024, 384, 128, 8, {}),
+])
+def test_edge_shapes_full_parity(T, d, F, E, k, kw):
+    w = synth.custom_workload("edge", T=T, d=d, ffn=F, E=E, k=k, seed=T + d, **kw)
+    li = synth.make_layer_inputs(w)
+    out = run_gpu(w, li)
+    print(check_full(w, li, out))
+
+
+def test_f32_gates_i32_idx_and_fold_collisions():
+    w = synth.custom_workload("fold", T=700, d=256, ffn=256, E=24, k=4, E_tgt=5, fold_mod=5, seed=11)
+    li = synth.make_layer_inputs(w)
+    out = run_gpu(w, li, gate_f32=True, idx_i32=True)
+    print(check_full(w, li, out))
+
+
+def test_dense_special_case_unit_gate():
+    """E=1, k=1, gate=1: the layer is a dense SwiGLU FFN."""
+    w = synth.custom_workload("dense", T=384, d=128, ffn=256, E=1, k=1, seed=5)
+    li = synth.make_layer_inputs(w)
+    li.gates = synth.f32_to_bf16_bits(np.ones((w.T, 1), dtype=np.float32))
+    out = run_gpu(w, li)
+    print(check_full(w, li, out))
+
+
+def test_plan_reuse_across_layers_and_determinism():
+    """One plan serves several forward/backward calls (all layers share the frozen router); results are bit-stable."""
+    from paper_2603_06626_b200 import binding
+    w = synth.WORKLOADS["tiny"]
+    li = synth.make_layer_inputs(w)
+    layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k)
+    idx, gates = to_dev(li.idx), bits_to_bf16(li.gates)
+    X, dY, W_gu, W_d = bits_to_bf16(li.X), bits_to_bf16(li.dY), bits_to_bf16(li.W_gu), bits_to_bf16(li.W_d)
+    layer.plan(idx)
+    Y1 = layer.forward(X, gates, W_gu, W_d).clone()
+    r1 = [t.clone() for t in layer.backward(dY, X, gates, W_gu, W_d)]
+    Y2 = layer.forward(X, gates, W_gu, W_d)
+    r2 = layer.backward(dY, X, gates, W_gu, W_d)
+    layer.check_status()
+    assert torch.equal(Y1, Y2)
+    for a, b in zip(r1, r2):
+        assert torch.equal(a, b)
+    layer.close()

@@ -1,0 +1,106 @@
+"""Plan kernels against the oracle: all four arrays bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import grouter_oracle as orc
+from paper_2603_06626_b200 import synth
+from tests.gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_plan(idx, fold_map, E_src, E_tgt, idx_i32=False):
+    from paper_2603_06626_b200 import binding
+    T, k = idx.shape
+    idx_np = idx.astype(np.int32) if idx_i32 else idx.astype(np.uint8)
+    layer = binding.GrouterLayer(T, 64, 64, E_src, k, E_tgt=E_tgt,
+                                 idx_dtype=binding.IDX_I32 if idx_i32 else binding.IDX_U8)
+    fm = None if fold_map is None else to_dev(fold_map.astype(np.int32))
+    out = layer.plan(to_dev(idx_np), fm)
+    st = layer.status()
+    res = [o.cpu().numpy() for o in out]
+    layer.close()
+    return res, st
+
+
+def _assert_equal(got, want):
+    for g, w, name in zip(got, want, ["counts", "offsets", "row_to_slot", "slot_to_row"]):
+        assert g.dtype == np.int32
+        assert np.array_equal(g, w), name
+
+
+@pytest.mark.parametrize("name", synth.WORKLOAD_ORDER)
+def test_plan_workloads_bit_exact(name):
+    w = synth.WORKLOADS[name]
+    idx, fm = synth.make_idx(w), synth.make_fold_map(w)
+    got, st = _run_plan(idx, fm, w.E_src, w.E_tgt)
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, fm, w.E_tgt))
+
+
+@pytest.mark.parametrize("T,k,E", [(1, 1, 1), (33, 1, 2), (1000, 3, 7), (4097, 2, 256), (777, 8, 128), (5000, 4, 1000)])
+def test_plan_ragged_sizes(T, k, E):
+    rng = np.random.default_rng(T + k + E)
+    idx = rng.integers(0, E, size=(T, k))
+    got, st = _run_plan(idx, None, E, E, idx_i32=E > 256)
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, None, E))
+
+
+def test_plan_degenerate_and_i32():
+    idx = np.full((3000, 2), 5)
+    got, st = _run_plan(idx, None, 9, 9)
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, None, 9))
+    rng = np.random.default_rng(3)
+    idx = rng.integers(0, 40, size=(2500, 4))
+    fm = rng.integers(0, 6, size=40)
+    for i32 in (False, True):
+        got, st = _run_plan(idx, fm, 40, 6, idx_i32=i32)
+        assert st == 0
+        _assert_equal(got, orc.plan(idx, fm, 6))
+
+
+def test_plan_reproducible_and_reusable():
+    from paper_2603_06626_b200 import binding
+    w = synth.WORKLOADS["skewed"]
+    idx = to_dev(synth.make_idx(w))
+    layer = binding.GrouterLayer(w.T, 64, 64, w.E_src, w.k)
+    first = [o.clone() for o in layer.plan(idx)]
+    for _ in range(3):
+        again = layer.plan(idx)
+        for a, b in zip(first, again):
+            assert torch.equal(a, b)
+    assert layer.status() == 0
+    layer.close()
+
+
+def test_plan_bad_index_sets_status_without_fault():
+    from paper_2603_06626_b200 import binding
+    idx = np.zeros((100, 2), dtype=np.uint8)
+    idx[7, 1] = 200                                  # >= E_src
+    got, st = _run_plan(idx, None, 8, 8)
+    assert st == -6
+    assert got[0].sum() == 200                        # every slot still counted (bad id treated as expert 0)
+    got, st = _run_plan(np.zeros((100, 2), dtype=np.uint8), None, 8, 8)
+    assert st == 0                                    # status is cleared by the previous read, and contexts are separate
+
+
+def test_host_side_errors():
+    from paper_2603_06626_b200 import binding
+    with pytest.raises(binding.GrouterError) as e:
+        binding.GrouterLayer(16, 60, 64, 4, 2)         # d % 8 != 0
+    assert e.value.code == -3
+    with pytest.raises(binding.GrouterError) as e:
+        binding.GrouterLayer(16, 64, 64, 300, 2)       # uint8 ids cannot address 300 experts
+    assert e.value.code == -3
+    layer = binding.GrouterLayer(16, 64, 64, 4, 2)
+    X = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda:0")
+    g = torch.zeros(16, 2, dtype=torch.bfloat16, device="cuda:0")
+    W_gu = torch.zeros(4, 128, 64, dtype=torch.bfloat16, device="cuda:0")
+    W_d = torch.zeros(4, 64, 64, dtype=torch.bfloat16, device="cuda:0")
+    with pytest.raises(binding.GrouterError) as e:
+        layer.forward(X, g, W_gu, W_d)                 # no plan yet
+    assert e.value.code == -4
+    layer.close()
