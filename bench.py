@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the routed SwiGLU expert layer under preemptive routing.
+
+A step is one pass of the whole hot path over one batch: routing-plan build,
+forward (gather, up/gate GEMM + SwiGLU, down GEMM, combine) and backward (dY
+gather, dH GEMM + SwiGLU backward + d-gate, three weight-gradient GEMMs, dX
+GEMM, dX reduce), all through the C ABI.  Metric: tokens per second of
+fwd+bwd.  One JSON line is printed by rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large] [--impl reference]
+
+N > 1 (launched with torch.distributed.run): every rank owns its own batch of
+the same shape (weak scaling over independent token shards, no collective on
+the data path; the weight-gradient all-reduce of data parallelism belongs to
+the optimizer step, outside the layer).  `--impl reference` times the fp64 CPU
+oracle on the host cores for the same metric.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2603_06626_b200 import synth  # noqa: E402
+
+METRIC = "moe_layer_fwd_bwd_tokens_per_sec"
+UNIT = "tokens/s"
+GEMM_SLOTS = ["gemm_up_swiglu", "gemm_down", "gemm_dH", "wgrad_down", "gemm_dX", "wgrad_gate_up"]
+MOVER_SLOTS = ["gather_X", "combine_Y", "gather_dY", "reduce_dX"]
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def kernel_work(w: synth.Workload):
+    """Algorithmic work per launch: FLOPs over valid routed rows only (padding earns nothing) for the
+    GEMMs; bytes (T + R) * d * 2 for the row movers; plan: ids read, two permutations written."""
+    R, d, F, T = w.R, w.d, w.ffn, w.T
+    dF = 2.0 * R * d * F
+    idb = 1 if w.E_src <= 256 else 4
+    return {
+        "gemm_up_swiglu": ("flop", 2 * dF), "gemm_down": ("flop", dF), "gemm_dH": ("flop", dF), "wgrad_down": ("flop", dF),
+        "gemm_dX": ("flop", 2 * dF), "wgrad_gate_up": ("flop", 2 * dF),
+        "gather_X": ("byte", (T + R) * d * 2.0), "combine_Y": ("byte", (T + R) * d * 2.0),
+        "gather_dY": ("byte", (T + R) * d * 2.0), "reduce_dX": ("byte", (T + R) * d * 2.0),
+        "plan_hist": ("byte", R * idb + 0.0), "plan_permute": ("byte", R * idb + 2.0 * R * 4),
+    }
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return out
+        sm, mx, pw = [], [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), power_w_max=max(pw), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample_tokens_per_sec(w: synth.Workload, li, n_tokens: int):
+    """The fp64 oracle, as it stands, on the first n_tokens tokens of the workload (full fwd + bwd incl. every
+    expert's weight gradients for those tokens).  Returns (tokens/s, seconds, threads)."""
+    from oracle import grouter_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    sub = slice(0, n_tokens)
+    X = synth.bf16_bits_to_f64(li.X[sub]); dY = synth.bf16_bits_to_f64(li.dY[sub]); gates = synth.bf16_bits_to_f64(li.gates[sub])
+    idx = li.idx[sub]
+    if li.W_gu is not None:
+        getter = lambda e: (synth.bf16_bits_to_f64(li.W_gu[e]), synth.bf16_bits_to_f64(li.W_d[e]))  # noqa: E731
+    else:
+        cache = {}
+
+        def getter(e):
+            if e not in cache:
+                cache[e] = (synth.expert_W_gu(w, e), synth.expert_W_d(w, e))
+            return synth.bf16_bits_to_f64(cache[e][0]), synth.bf16_bits_to_f64(cache[e][1])
+        used = np.unique(orc.fold_ids(idx, li.fold_map))
+        for e in used:           # draw the weights before the clock starts
+            getter(int(e))
+    weights = orc.Weights(getter=getter, ffn=w.ffn)
+    used = [int(e) for e in np.unique(orc.fold_ids(idx, li.fold_map))]
+    t0 = time.perf_counter()
+    orc.moe_forward(X, idx, gates, weights, w.E_tgt, li.fold_map)
+    orc.moe_backward(dY, X, idx, gates, weights, w.E_tgt, li.fold_map, experts=used)
+    dt = time.perf_counter() - t0
+    return n_tokens / dt, dt, threads
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle timed on the host cores, same metric and workload config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = synth.WORKLOADS[args.workload]
+    li = synth.make_layer_inputs(w, with_weights=False)
+    n = args.ref_tokens
+    times = []
+    threads = 1
+    for i in range(args.warmup + args.steps):
+        _, dt, threads = oracle_sample_tokens_per_sec(w, li, n)
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = n * len(times) / total
+    sample = f"first {n} tokens of the workload per step (all their experts, fwd + full bwd), fp64 numpy"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, args.gpus),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w: synth.Workload, n_gpus: int):
+    return {"workload": w.name, "T": w.T, "d": w.d, "ffn": w.ffn, "E_src": w.E_src, "E_tgt": w.E_tgt, "k": w.k, "load": w.load,
+            "zipf_s": w.zipf_s, "tokens_per_gpu": w.T, "global_tokens": w.T * n_gpus, "parallelism": f"dp{n_gpus}",
+            "l2": "working set (weights + expert-ordered activations, several GB) exceeds the 126 MB L2"
+            if w.name in ("skewed", "large", "fine_fold", "small") else "fits L2: flushed between steps"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="large", choices=list(synth.WORKLOADS))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--ref-tokens", type=int, default=2, help="tokens per step of the reference arm's oracle sample")
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=48)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_06626_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    warm = max(args.warmup, 3)
+
+    base = synth.WORKLOADS[args.workload]
+    w = synth.reseeded(base, base.seed + 1000 * rank) if rank else base
+    li = synth.make_layer_inputs(w, threads=min(16, os.cpu_count() or 1))
+
+    def bf16(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt, device=str(dev), host_staging=not args.no_e2e)
+    idx = torch.from_numpy(li.idx).to(dev)
+    fm = None if li.fold_map is None else torch.from_numpy(li.fold_map).to(dev)
+    gates, X, dY = bf16(li.gates), bf16(li.X), bf16(li.dY)
+    W_gu, W_d = bf16(li.W_gu), bf16(li.W_d)
+    Y, dX = torch.empty_like(X), torch.empty_like(X)
+    dW_gu = torch.empty(W_gu.shape, dtype=torch.float32, device=dev)
+    dW_d = torch.empty(W_d.shape, dtype=torch.float32, device=dev)
+    dgates = torch.empty((w.T, w.k), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if w.name == "tiny" else None
+
+    def step():
+        if flush is not None:
+            flush.zero_()
+        layer.plan(idx, fm)
+        layer.forward(X, gates, W_gu, W_d, Y)
+        layer.backward(dY, X, gates, W_gu, W_d, dX, dW_gu, dW_d, dgates)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for _ in range(warm):
+        step()
+    layer.check_status()
+    barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    layer.timing_enable(12 * args.steps)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else None
+    per_kernel = layer.timing_read()
+    layer.timing_enable(0)
+    layer.check_status()
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * w.T / (ms_step * 1e-3)
+
+    # ---- end to end: host buffers in, host results out, every step ----
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()  # noqa: E731
+        idx_h, gates_h = pin(li.idx), pin(li.gates.view(np.int16))
+        X_h, dY_h = pin(li.X.view(np.int16)), pin(li.dY.view(np.int16))
+        Y_h = torch.empty((w.T, w.d), dtype=torch.int16).pin_memory()
+        dX_h = torch.empty((w.T, w.d), dtype=torch.int16).pin_memory()
+        dg_h = torch.empty((w.T, w.k), dtype=torch.float32).pin_memory()
+
+        def e2e_step():
+            layer.step_host(idx_h, gates_h, X_h, dY_h, fm, W_gu, W_d, Y_h, dX_h, dg_h, dW_gu, dW_d)
+            torch.cuda.current_stream().synchronize()     # the step's results are read on the host
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record()
+        torch.cuda.synchronize()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        layer.check_status()
+        h2d = idx_h.numel() * idx_h.element_size() + gates_h.numel() * 2 + X_h.numel() * 2 + dY_h.numel() * 2
+        d2h = Y_h.numel() * 2 + dX_h.numel() * 2 + dg_h.numel() * 4
+        e2e = {"value": world * w.T / (ms_e2e / args.e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
+               "note": "idx, gates, X, dY copied from pinned host memory and Y, dX, dgates copied back every step "
+                       "(grouter_moe_step_host); weights and weight gradients stay on the device"}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel, and the per-kernel table ----
+    peaks, peak_src = load_peaks()
+    work = kernel_work(w)
+    kernels = {}
+    for name, (ms, n) in per_kernel.items():
+        if n == 0:
+            continue
+        kind, amount = work[name]
+        avg_s = ms / n * 1e-3
+        ent = {"launches": n, "avg_ms": ms / n, "share": ms / sum(v[0] for v in per_kernel.values())}
+        if kind == "flop":
+            ent["tflops"] = amount / avg_s / 1e12
+            ent["frac_of_sustained"] = ent["tflops"] / peaks["bf16_tflops_sustained"]
+            ent["frac_of_burst"] = ent["tflops"] / peaks["bf16_tflops"]
+        else:
+            ent["gbs"] = amount / avg_s / 1e9
+            ent["frac_of_hbm"] = ent["gbs"] / peaks["hbm_gbs"]
+        kernels[name] = ent
+    dom = max(GEMM_SLOTS, key=lambda k: per_kernel[k][0])
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(w.name, {}).get(dom)
+    roofline = {"kernel": dom, "bound": "tensor", "achieved": kernels[dom]["tflops"], "peak": peaks["bf16_tflops_sustained"],
+                "unit": "TFLOP/s", "frac": kernels[dom]["tflops"] / peaks["bf16_tflops_sustained"], "traffic": traffic,
+                "peak_source": f"{peak_src} cuBLAS bf16, sustained (kernel timed inside a long step); burst peak "
+                               f"{peaks['bf16_tflops']} gives frac {kernels[dom]['tflops'] / peaks['bf16_tflops']:.3f}"}
+    gemm_ms = sum(per_kernel[k][0] for k in GEMM_SLOTS)
+    gemm_flops = sum(work[k][1] * per_kernel[k][1] for k in GEMM_SLOTS)
+    summary = {"all_gemms_tflops": gemm_flops / (gemm_ms * 1e-3) / 1e12,
+               "all_gemms_frac_of_burst": gemm_flops / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+               "step_flops": 18.0 * w.d * w.ffn * w.R}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": workload_config(base, world), "clocks": clocks,
+        "gpu_launches": int(sum(v[1] for v in per_kernel.values())), "roofline": roofline, "kernels": kernels, "gemm_summary": summary,
+        "load_stats": synth.load_stats(li.idx, li.fold_map, w.E_tgt),
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        v, dt, threads = oracle_sample_tokens_per_sec(w, li, args.cpu_baseline_tokens)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
+                                "sample": f"first {args.cpu_baseline_tokens} tokens of the workload (all their experts, fwd + full bwd), "
+                                          "fp64 numpy oracle"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

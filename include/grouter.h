@@ -139,6 +139,19 @@ int grouter_status(grouter_ctx* ctx, void* stream);
 
 const char* grouter_strerror(int code);
 
+/* Per-kernel device timing (measurement aid; no counterpart in the paper).
+ * grouter_timing_enable(ctx, n) creates n CUDA event pairs (host call, allocates;
+ * n = 0 frees them and switches timing off).  While enabled, every kernel launch
+ * of plan/fwd/bwd is bracketed by an event pair on the caller's stream until the
+ * pool is used up.  grouter_timing_read synchronises `stream`, adds up the
+ * elapsed milliseconds and launch counts per kernel slot, and empties the pool.
+ * Slots: 0 plan_hist, 1 plan_permute, 2 gather_X, 3 gemm_up_swiglu, 4 gemm_down,
+ * 5 combine_Y, 6 gather_dY, 7 gemm_dH, 8 wgrad_down, 9 gemm_dX, 10 wgrad_gate_up,
+ * 11 reduce_dX.   total_ms, launches: HOST arrays of GROUTER_NUM_KERNELS entries. */
+#define GROUTER_NUM_KERNELS 12
+int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records);
+int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t* launches);
+
 /* Component check of the tensor-core core used by every grouped GEMM (no
  * counterpart in the paper): C[M,N] (f32) = A * B with bf16 operands.
  *   a_mn_major == 0: A stored [M,K] (K contiguous); != 0: A stored [K,M].

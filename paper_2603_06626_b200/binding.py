@@ -19,7 +19,9 @@ GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
-           "grouter_dense_gemm"]
+           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read"]
+KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
+                "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX"]
 
 
 class GrouterDims(ctypes.Structure):
@@ -68,6 +70,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_strerror.restype = ctypes.c_char_p
     lib.grouter_dense_gemm.argtypes = [vp, ctypes.c_int, vp, ctypes.c_int, f32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
     lib.grouter_dense_gemm.restype = ctypes.c_int
+    lib.grouter_timing_enable.argtypes = [vp, ctypes.c_int32]
+    lib.grouter_timing_enable.restype = ctypes.c_int
+    lib.grouter_timing_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
+    lib.grouter_timing_read.restype = ctypes.c_int
     if path == _build.LIB:
         _lib = lib
     return lib
@@ -161,6 +167,17 @@ class GrouterLayer:
         _check(self.lib.grouter_moe_step_host(self.ctx, _ptr(idx_h), _ptr(gates_h), _ptr(X_h), _ptr(dY_h), _ptr(fold_map), _ptr(W_gu),
                                               _ptr(W_d), _ptr(Y_h), _ptr(dX_h), _ptr(dgates_h), _ptr(dW_gu), _ptr(dW_d),
                                               _ptr(self.workspace), _stream()), "grouter_moe_step_host")
+
+    def timing_enable(self, n_records: int) -> None:
+        _check(self.lib.grouter_timing_enable(self.ctx, n_records), "grouter_timing_enable")
+
+    def timing_read(self):
+        """-> {kernel name: (total ms, launches)} since the last read; synchronises the current stream."""
+        n = len(KERNEL_SLOTS)
+        ms = (ctypes.c_float * n)()
+        cnt = (ctypes.c_int32 * n)()
+        _check(self.lib.grouter_timing_read(self.ctx, _stream(), ms, cnt), "grouter_timing_read")
+        return {KERNEL_SLOTS[i]: (float(ms[i]), int(cnt[i])) for i in range(n)}
 
     def status(self) -> int:
         """Synchronises the current stream; returns 0 or a negative GROUTER_ERR_* device status."""

@@ -52,6 +52,36 @@ Staging staging_layout(const grouter_dims& dm) {
   return s;
 }
 
+// Brackets one kernel launch with an event pair while timing is enabled.
+struct Timed {
+  grouter_ctx* c;
+  cudaStream_t st;
+  int i;
+  Timed(grouter_ctx* ctx, int slot, cudaStream_t s) : c(ctx), st(s), i(-1) {
+    if (c->ev_cap > 0 && c->ev_used < c->ev_cap) {
+      i = c->ev_used++;
+      c->ev_slot[i] = slot;
+      cudaEventRecord(c->ev_start[i], st);
+    }
+  }
+  ~Timed() {
+    if (i >= 0) cudaEventRecord(c->ev_stop[i], st);
+  }
+};
+
+void free_events(grouter_ctx* c) {
+  for (int i = 0; i < c->ev_cap; ++i) {
+    cudaEventDestroy(c->ev_start[i]);
+    cudaEventDestroy(c->ev_stop[i]);
+  }
+  delete[] c->ev_start;
+  delete[] c->ev_stop;
+  delete[] c->ev_slot;
+  c->ev_start = c->ev_stop = nullptr;
+  c->ev_slot = nullptr;
+  c->ev_cap = c->ev_used = 0;
+}
+
 }  // namespace
 
 namespace grouter {
@@ -126,6 +156,9 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->max_m_tiles = (int)(c->R_pad_max / ROW_TILE);
   c->geom = plan_geom(c->R);
   c->planned = c->forwarded = false;
+  c->ev_start = c->ev_stop = nullptr;
+  c->ev_slot = nullptr;
+  c->ev_cap = c->ev_used = 0;
   const int E = dims->E_tgt;
   size_t off = 0;
   auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
@@ -158,6 +191,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
 
 void grouter_destroy(grouter_ctx* ctx) {
   if (!ctx) return;
+  free_events(ctx);
   if (ctx->d_block) cudaFree(ctx->d_block);
   delete ctx;
 }
@@ -169,8 +203,11 @@ int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int
       (fold_map && !aligned16(fold_map)))
     return GROUTER_ERR_MISALIGNED;
   if (!fold_map && ctx->dims.E_src != ctx->dims.E_tgt) return GROUTER_ERR_INVALID_ARG;
-  if (launch_plan(ctx, idx, fold_map, counts, offsets, row_to_slot, slot_to_row, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-    return GROUTER_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  for (int phase = 0; phase < 2; ++phase) {
+    Timed tm(ctx, phase, st);
+    if (launch_plan(ctx, phase, idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
   ctx->planned = true;
   ctx->forwarded = false;
   return GROUTER_OK;
@@ -185,10 +222,22 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
   if (!ctx->planned) return GROUTER_ERR_INVALID_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Workspace ws = carve_workspace(ctx->dims, ctx->R_pad_max, workspace);
-  if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(X), ws.Xp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_grouped_gemm(ctx, MODE_UP, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_grouped_gemm(ctx, MODE_DOWN, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  {
+    Timed tm(ctx, 2, st);
+    if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(X), ws.Xp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 3, st);
+    if (launch_grouped_gemm(ctx, MODE_UP, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 4, st);
+    if (launch_grouped_gemm(ctx, MODE_DOWN, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 5, st);
+    if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
   ctx->forwarded = true;
   return GROUTER_OK;
 }
@@ -203,13 +252,31 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Workspace ws = carve_workspace(ctx->dims, ctx->R_pad_max, workspace);
   const int n_part = (ctx->dims.ffn + 255) / 256;
-  if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(dY), ws.dYp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_grouped_gemm(ctx, MODE_DH, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_grouped_gemm(ctx, MODE_WGRAD_D, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_grouped_gemm(ctx, MODE_DX, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_grouped_gemm(ctx, MODE_WGRAD_GU, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(dX), ws.dgate_part, n_part, dgates, st) != cudaSuccess)
-    return GROUTER_ERR_CUDA;
+  {
+    Timed tm(ctx, 6, st);
+    if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(dY), ws.dYp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 7, st);
+    if (launch_grouped_gemm(ctx, MODE_DH, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 8, st);
+    if (launch_grouped_gemm(ctx, MODE_WGRAD_D, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 9, st);
+    if (launch_grouped_gemm(ctx, MODE_DX, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 10, st);
+    if (launch_grouped_gemm(ctx, MODE_WGRAD_GU, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 11, st);
+    if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(dX), ws.dgate_part, n_part, dgates, st) != cudaSuccess)
+      return GROUTER_ERR_CUDA;
+  }
   return GROUTER_OK;
 }
 
@@ -255,6 +322,43 @@ int grouter_status(grouter_ctx* ctx, void* stream) {
     if (h & STATUS_TIMEOUT) return GROUTER_ERR_TIMEOUT;
     return GROUTER_ERR_BAD_INDEX;
   }
+  return GROUTER_OK;
+}
+
+int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records) {
+  if (!ctx || n_records < 0) return GROUTER_ERR_INVALID_ARG;
+  free_events(ctx);
+  if (n_records == 0) return GROUTER_OK;
+  ctx->ev_start = new (std::nothrow) cudaEvent_t[n_records];
+  ctx->ev_stop = new (std::nothrow) cudaEvent_t[n_records];
+  ctx->ev_slot = new (std::nothrow) int[n_records];
+  if (!ctx->ev_start || !ctx->ev_stop || !ctx->ev_slot) return GROUTER_ERR_INVALID_ARG;
+  for (int i = 0; i < n_records; ++i) {
+    if (cudaEventCreate(&ctx->ev_start[i]) != cudaSuccess || cudaEventCreate(&ctx->ev_stop[i]) != cudaSuccess) {
+      ctx->ev_cap = i;
+      free_events(ctx);
+      return GROUTER_ERR_CUDA;
+    }
+  }
+  ctx->ev_cap = n_records;
+  ctx->ev_used = 0;
+  return GROUTER_OK;
+}
+
+int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t* launches) {
+  if (!ctx || !total_ms || !launches) return GROUTER_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return GROUTER_ERR_CUDA;
+  for (int k = 0; k < GROUTER_NUM_KERNELS; ++k) {
+    total_ms[k] = 0.f;
+    launches[k] = 0;
+  }
+  for (int i = 0; i < ctx->ev_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->ev_start[i], ctx->ev_stop[i]) != cudaSuccess) return GROUTER_ERR_CUDA;
+    total_ms[ctx->ev_slot[i]] += ms;
+    launches[ctx->ev_slot[i]] += 1;
+  }
+  ctx->ev_used = 0;
   return GROUTER_OK;
 }
 

@@ -63,6 +63,12 @@ struct grouter_ctx {
   bool planned;
   bool forwarded;
   int num_sms;
+  // optional per-kernel timing (event pool)
+  cudaEvent_t* ev_start;
+  cudaEvent_t* ev_stop;
+  int* ev_slot;
+  int ev_cap;
+  int ev_used;
 };
 
 namespace grouter {
@@ -82,7 +88,7 @@ struct Workspace {
 Workspace carve_workspace(const grouter_dims& dm, int64_t R_pad_max, void* base);
 
 // ---- launchers (each returns a cudaError_t from the launch) ----
-cudaError_t launch_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
                         int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st);
 
 // dst[prow,:] = src[slot/k,:] for every routed slot; pad rows zero-filled.

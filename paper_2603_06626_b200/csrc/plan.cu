@@ -216,26 +216,28 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_permute_kernel(const IdxT* 
 }
 
 template <typename IdxT>
-static cudaError_t launch_plan_t(grouter_ctx* ctx, const IdxT* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
-                                 int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
+static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, const int32_t* fold_map, int32_t* counts,
+                                 int32_t* offsets, int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
   const int R = (int)ctx->R, E = dm.E_tgt;
   const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
-  const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 3 * E + 3) ? PLAN_WARPS * E : 3 * E + 3);
-  const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
-  plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
-  cudaError_t err = cudaGetLastError();
-  if (err != cudaSuccess) return err;
-  plan_permute_kernel<IdxT><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, offsets, row_to_slot,
-                                                             slot_to_row);
+  if (phase == 0) {
+    const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 3 * E + 3) ? PLAN_WARPS * E : 3 * E + 3);
+    plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
+  } else {
+    const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
+    plan_permute_kernel<IdxT><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, offsets,
+                                                               row_to_slot, slot_to_row);
+  }
   return cudaGetLastError();
 }
 
-cudaError_t launch_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
+// phase 0: histogram + scans (counts, offsets, padded layout); phase 1: stable permutation.
+cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
                         int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
   if (ctx->dims.idx_dtype == GROUTER_IDX_U8)
-    return launch_plan_t<uint8_t>(ctx, (const uint8_t*)idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st);
-  return launch_plan_t<int32_t>(ctx, (const int32_t*)idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st);
+    return launch_plan_t<uint8_t>(ctx, phase, (const uint8_t*)idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st);
+  return launch_plan_t<int32_t>(ctx, phase, (const int32_t*)idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st);
 }
 
 }  // namespace grouter

@@ -183,18 +183,35 @@ class LayerInputs:
     extra: dict = field(default_factory=dict)
 
 
-def make_layer_inputs(w: Workload, with_weights: bool = True) -> LayerInputs:
+def make_layer_inputs(w: Workload, with_weights: bool = True, threads: int = 0) -> LayerInputs:
     """All inputs of one fwd+bwd step.  Weights can be skipped and drawn per
-    expert later with `expert_W_gu` / `expert_W_d` (same bits)."""
+    expert later with `expert_W_gu` / `expert_W_d` (same bits).  `threads` > 1
+    draws the experts' weights in parallel (each expert has its own stream, so
+    the bits do not depend on it)."""
     li = LayerInputs(w=w, X=make_tokens(w), dY=make_dY(w), idx=make_idx(w), gates=make_gates(w),
                      fold_map=make_fold_map(w))
     if with_weights:
         li.W_gu = np.empty((w.E_tgt, 2 * w.ffn, w.d), dtype=np.uint16)
         li.W_d = np.empty((w.E_tgt, w.d, w.ffn), dtype=np.uint16)
-        for e in range(w.E_tgt):
+
+        def fill(e):
             li.W_gu[e] = expert_W_gu(w, e)
             li.W_d[e] = expert_W_d(w, e)
+
+        if threads > 1:
+            from concurrent.futures import ThreadPoolExecutor
+            with ThreadPoolExecutor(max_workers=threads) as pool:
+                list(pool.map(fill, range(w.E_tgt)))
+        else:
+            for e in range(w.E_tgt):
+                fill(e)
     return li
+
+
+def reseeded(w: Workload, seed: int) -> Workload:
+    """Same shapes and load recipe, different random streams (one per data-parallel rank)."""
+    from dataclasses import replace
+    return replace(w, seed=int(seed))
 
 
 def custom_workload(name: str, T: int, d: int, ffn: int, E: int, k: int, *, load: str = "uniform",
