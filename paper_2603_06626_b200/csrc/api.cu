@@ -92,7 +92,7 @@ Workspace carve_workspace(const grouter_dims& dm, int64_t Rp, void* base) {
   auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
   const size_t rd = (size_t)Rp * dm.d * 2, rf = (size_t)Rp * dm.ffn * 2;
   const size_t oXp = take(rd), oG = take(rf), oU = take(rf), oH = take(rf), oO = take(rd), odY = take(rd), odGU = take(2 * rf);
-  const size_t oPart = take((size_t)((dm.ffn + 255) / 256) * Rp * 4);
+  const size_t oPart = take((size_t)(2 * ((dm.ffn + 255) / 256)) * Rp * 4);
   w.bytes = off;
   if (b) {
     w.Xp = reinterpret_cast<__nv_bfloat16*>(b + oXp);
@@ -251,7 +251,7 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
   if (!ctx->planned || !ctx->forwarded) return GROUTER_ERR_INVALID_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Workspace ws = carve_workspace(ctx->dims, ctx->R_pad_max, workspace);
-  const int n_part = (ctx->dims.ffn + 255) / 256;
+  const int n_part = 2 * ((ctx->dims.ffn + 255) / 256);  // two column halves per 256-wide tile
   {
     Timed tm(ctx, 6, st);
     if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(dY), ws.dYp, st) != cudaSuccess) return GROUTER_ERR_CUDA;

@@ -82,7 +82,7 @@ struct Workspace {
   __nv_bfloat16* O;     // [R_pad_max, d]   expert outputs (fwd) / dXp (bwd)
   __nv_bfloat16* dYp;   // [R_pad_max, d]   gathered upstream gradient
   __nv_bfloat16* dGU;   // [R_pad_max, 2F]  [dG | dU]
-  float* dgate_part;    // [ceil(F/256), R_pad_max] partial row sums for d-gate
+  float* dgate_part;    // [2*ceil(F/256), R_pad_max] partial row sums for d-gate
   size_t bytes;
 };
 Workspace carve_workspace(const grouter_dims& dm, int64_t R_pad_max, void* base);

@@ -12,7 +12,7 @@
 // Tile: 128 x 256 x 64 per CTA, one CTA per SM.  Warp 0 issues TMA tile loads
 // (128-byte swizzle) into a 4-stage shared-memory ring; warp 1 issues
 // tcgen05.mma (M=128, N=256, K=16) into one of two 256-column TMEM
-// accumulators; warps 2-5 drain the other accumulator with tcgen05.ld and run
+// accumulators; warps 2-9 drain the other accumulator with tcgen05.ld and run
 // the fused epilogue, so the epilogue of tile i overlaps the main loop of tile
 // i+1.  Operands may be K-major (rows of the stored matrix run along K) or
 // MN-major (rows run along M/N); both are described to the MMA by
@@ -31,7 +31,8 @@ constexpr int A_BYTES = BM * BK * 2;            // 16 KB
 constexpr int B_BYTES = BN * BK * 2;            // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 48 KB
 constexpr int ATOM_BYTES = 64 * BK * 2;         // one 64x64 bf16 box = 8 KB
-constexpr int GEMM_THREADS = 192;
+constexpr int EPI_WARPS = 8;                    // two warps per TMEM lane quadrant, each takes half of the columns
+constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = 512;
 
@@ -206,7 +207,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), 4);
+      ptx::mbar_init(tempty_bar(a), EPI_WARPS);
     }
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
@@ -308,8 +309,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     __syncwarp();
   } else {
-    // ===================== epilogue (warps 2..5) =====================
+    // ===================== epilogue (warps 2..9) =====================
     const int quad = warp & 3;            // TMEM lane quadrant this warp may read
+    const int half = (warp - 2) >> 2;     // which half of the tile's columns this warp drains
     const int r = quad * 32 + lane;       // row of the tile owned by this thread
     int acc = 0;
     uint32_t acc_ph = 0;
@@ -324,7 +326,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const size_t prow = (size_t)ti.row0 + r;
         const float g = gate_of_row(p, (int)prow);
         const size_t o = prow * p.F + ti.col0;
-        for (int c = 0; c < 4; ++c) {
+        for (int c = half * 2; c < half * 2 + 2; ++c) {
           const int n_left = ti.n_valid - c * 32;
           if (n_left <= 0) break;
           uint32_t rg[32], ru[32];
@@ -336,7 +338,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int i = 0; i < 32; ++i) {
             vg[i] = __uint_as_float(rg[i]);
             vu[i] = __uint_as_float(ru[i]);
-            const float sg = 1.f / (1.f + __expf(-vg[i]));
+            const float sg = __fdividef(1.f, 1.f + __expf(-vg[i]));
             vh[i] = g * vg[i] * sg * vu[i];
           }
           store_row32_bf16(p.out_b0 + o + c * 32, vg, n_left);
@@ -346,7 +348,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       } else if (MODE == MODE_DOWN || MODE == MODE_DX) {
         const size_t prow = (size_t)ti.row0 + r;
         const size_t o = prow * p.d + ti.col0;
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
           const int n_left = ti.n_valid - c * 32;
           if (n_left <= 0) break;
           uint32_t ra[32];
@@ -363,9 +365,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const size_t gi = prow * p.F + ti.col0;
         const size_t oi = prow * 2 * (size_t)p.F + ti.col0;
         float dgate = 0.f;
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
           const int n_left = ti.n_valid - c * 32;
           if (n_left <= 0) break;
+          // saved pre-activations of this chunk: issue the loads before waiting on TMEM
+          uint4 g4[4], u4[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (q * 8 < n_left) {
+              g4[q] = *reinterpret_cast<const uint4*>(p.in_G + gi + c * 32 + q * 8);
+              u4[q] = *reinterpret_cast<const uint4*>(p.in_U + gi + c * 32 + q * 8);
+            }
+          }
           uint32_t ra[32];
           ptx::tmem_ld32(t_row + c * 32, ra);
           ptx::tmem_ld_wait();
@@ -374,12 +385,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int q = 0; q < 4; ++q) {
             if (q * 8 < n_left) {
               float fg[8], fu[8];
-              unpack8(*reinterpret_cast<const uint4*>(p.in_G + gi + c * 32 + q * 8), fg);
-              unpack8(*reinterpret_cast<const uint4*>(p.in_U + gi + c * 32 + q * 8), fu);
+              unpack8(g4[q], fg);
+              unpack8(u4[q], fu);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const float dA = __uint_as_float(ra[q * 8 + i]);
-                const float sg = 1.f / (1.f + __expf(-fg[i]));
+                const float sg = __fdividef(1.f, 1.f + __expf(-fg[i]));
                 const float si = fg[i] * sg;            // silu(G)
                 dgate += dA * si * fu[i];                // <dA, H>
                 const float dH = g * dA;
@@ -395,7 +406,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           store_row32_bf16(p.out_b0 + oi + p.F + c * 32, vdu, n_left);
         }
         const int nt = ti.col0 / BN;
-        p.out_f[(size_t)nt * p.R_pad_max + prow] = dgate;
+        p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + prow] = dgate;
       } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile store
         float* C = p.out_f;
         size_t ld;
@@ -407,7 +418,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         const bool row_ok = r < ti.m_valid;
         float* crow = C + ((size_t)ti.row0 + r) * ld + ti.col0;
-        for (int c = 0; c < BN / 32; ++c) {
+        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
           const int n_left = ti.n_valid - c * 32;
           if (n_left <= 0) break;
           uint32_t ra[32];
