@@ -33,7 +33,8 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 48 KB
 constexpr int ATOM_BYTES = 64 * BK * 2;         // one 64x64 bf16 box = 8 KB
 constexpr int EPI_WARPS = 8;                    // two warps per TMEM lane quadrant, each takes half of the columns
 constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int EPI_STAGE_BYTES = 32 * 128;       // per epilogue warp: 32 rows x 128 bytes
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct GemmParams {
@@ -49,12 +50,9 @@ struct GemmParams {
   const int32_t* prow_to_slot;
   const void* gates;
   int32_t gate_is_f32;
-  __nv_bfloat16* out_b0;       // UP: G      DOWN/DX: O / dXp     DH: dGU
-  __nv_bfloat16* out_b1;       // UP: U
-  __nv_bfloat16* out_b2;       // UP: H'
   const __nv_bfloat16* in_G;   // DH
   const __nv_bfloat16* in_U;   // DH
-  float* out_f;                // WGRAD / DENSE: C ; DH: dgate_part
+  float* out_f;                // DH: dgate_part
   int32_t* status;
 };
 
@@ -167,27 +165,15 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
   }
 }
 
-// Stores 32 consecutive bf16 of one row (fp32 in v), 16 bytes at a time, columns >= n_left masked off.
-__device__ __forceinline__ void store_row32_bf16(__nv_bfloat16* dst, const float (&v)[32], int n_left) {
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    if (q * 8 < n_left) {
-      uint4 o;
-      o.x = pack_bf16(v[q * 8 + 0], v[q * 8 + 1]);
-      o.y = pack_bf16(v[q * 8 + 2], v[q * 8 + 3]);
-      o.z = pack_bf16(v[q * 8 + 4], v[q * 8 + 5]);
-      o.w = pack_bf16(v[q * 8 + 6], v[q * 8 + 7]);
-      *reinterpret_cast<uint4*>(dst + q * 8) = o;
-    }
-  }
-}
-
 template <int MODE, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
-grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
+                    const __grid_constant__ CUtensorMap tmC2, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + STAGES * STAGE_BYTES;
+  const uint32_t stage_base = smem_base + STAGES * STAGE_BYTES;          // epilogue staging, 4 KB per warp
+  const uint32_t bar_base = stage_base + EPI_WARPS * EPI_STAGE_BYTES;
   // barriers (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
@@ -212,6 +198,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    ptx::prefetch_tensormap(&tmC0);
+    if (MODE == MODE_UP || MODE == MODE_DH) ptx::prefetch_tensormap(&tmC1);
+    if (MODE == MODE_UP) ptx::prefetch_tensormap(&tmC2);
   }
   if (warp == 1) {
     ptx::tmem_alloc(ptx::smem_u32(&s_tmem_base), TMEM_COLS);
@@ -310,9 +299,45 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncwarp();
   } else {
     // ===================== epilogue (warps 2..9) =====================
+    // Thread (quad, lane) owns tile row quad*32 + lane; the warp drains the 128 accumulator columns of
+    // its half.  Results go through a warp-private 32-row x 128-byte staging block in shared memory
+    // (128-byte swizzle, conflict-free) and leave as TMA tile stores: full 128-byte lines, clipped at
+    // the tensor bounds, so no store is masked by hand.
     const int quad = warp & 3;            // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;     // which half of the tile's columns this warp drains
     const int r = quad * 32 + lane;       // row of the tile owned by this thread
+    const uint32_t stage_buf = stage_base + (uint32_t)(warp - 2) * EPI_STAGE_BYTES;
+    const uint32_t my_row = stage_buf + (uint32_t)lane * 128u;
+    const uint32_t sw = (uint32_t)(lane & 7);
+    auto stage_open = [&]() {             // the previous store out of this block has been read
+      if (lane == 0) ptx::bulk_wait_read0();
+      __syncwarp();
+    };
+    auto stage_put = [&](int q, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {  // 16-byte unit q of this row
+      ptx::st_shared_v4(my_row + (((uint32_t)q ^ sw) << 4), a, b, c, d);
+    };
+    auto stage_put_bf16 = [&](int q0, const float (&v)[32]) {  // 32 fp32 -> 4 units of 8 bf16
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        stage_put(q0 + q, pack_bf16(v[q * 8 + 0], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
+                  pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
+    };
+    auto stage_send_2d = [&](const CUtensorMap* tm, int x, int y) {
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::tma_store_2d(tm, stage_buf, x, y);
+        ptx::bulk_commit();
+      }
+    };
+    auto stage_send_3d = [&](const CUtensorMap* tm, int x, int y, int z) {
+      ptx::fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::tma_store_3d(tm, stage_buf, x, y, z);
+        ptx::bulk_commit();
+      }
+    };
     int acc = 0;
     uint32_t acc_ph = 0;
     for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
@@ -321,122 +346,138 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       ptx::tc_fence_after();
       const uint32_t t_row = tmem_base + (uint32_t)acc * BN + ((uint32_t)(quad * 32) << 16);
       const bool have_acc = ti.num_k > 0;
+      const int y0 = ti.row0 + quad * 32;  // first output row of this warp's block
 
       if (MODE == MODE_UP) {
-        const size_t prow = (size_t)ti.row0 + r;
-        const float g = gate_of_row(p, (int)prow);
-        const size_t o = prow * p.F + ti.col0;
-        for (int c = half * 2; c < half * 2 + 2; ++c) {
-          const int n_left = ti.n_valid - c * 32;
-          if (n_left <= 0) break;
-          uint32_t rg[32], ru[32];
-          ptx::tmem_ld32(t_row + c * 32, rg);
-          ptx::tmem_ld32(t_row + 128 + c * 32, ru);
-          ptx::tmem_ld_wait();
-          float vg[32], vu[32], vh[32];
+        // accumulator columns 0..127 = gate, 128..255 = up, for F-columns col0..col0+127; this warp: 64 of them
+        if (ti.n_valid - half * 64 > 0) {
+          const float g = gate_of_row(p, ti.row0 + r);
+          uint32_t pg[32], pu[32], ph[32];   // packed bf16 pairs: 64 columns each
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            vg[i] = __uint_as_float(rg[i]);
-            vu[i] = __uint_as_float(ru[i]);
-            const float sg = __fdividef(1.f, 1.f + __expf(-vg[i]));
-            vh[i] = g * vg[i] * sg * vu[i];
+          for (int cc = 0; cc < 2; ++cc) {
+            uint32_t rg[32], ru[32];
+            ptx::tmem_ld32(t_row + half * 64 + cc * 32, rg);
+            ptx::tmem_ld32(t_row + 128 + half * 64 + cc * 32, ru);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float g0 = __uint_as_float(rg[i]), g1 = __uint_as_float(rg[i + 1]);
+              const float u0 = __uint_as_float(ru[i]), u1 = __uint_as_float(ru[i + 1]);
+              const float s0 = __fdividef(1.f, 1.f + __expf(-g0)), s1 = __fdividef(1.f, 1.f + __expf(-g1));
+              pg[cc * 16 + i / 2] = pack_bf16(g0, g1);
+              pu[cc * 16 + i / 2] = pack_bf16(u0, u1);
+              ph[cc * 16 + i / 2] = pack_bf16(g * g0 * s0 * u0, g * g1 * s1 * u1);
+            }
           }
-          store_row32_bf16(p.out_b0 + o + c * 32, vg, n_left);
-          store_row32_bf16(p.out_b1 + o + c * 32, vu, n_left);
-          store_row32_bf16(p.out_b2 + o + c * 32, vh, n_left);
+          const int x = ti.col0 + half * 64;
+          stage_open();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) stage_put(q, pg[q * 4], pg[q * 4 + 1], pg[q * 4 + 2], pg[q * 4 + 3]);
+          stage_send_2d(&tmC0, x, y0);
+          stage_open();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) stage_put(q, pu[q * 4], pu[q * 4 + 1], pu[q * 4 + 2], pu[q * 4 + 3]);
+          stage_send_2d(&tmC1, x, y0);
+          stage_open();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) stage_put(q, ph[q * 4], ph[q * 4 + 1], ph[q * 4 + 2], ph[q * 4 + 3]);
+          stage_send_2d(&tmC2, x, y0);
         }
       } else if (MODE == MODE_DOWN || MODE == MODE_DX) {
-        const size_t prow = (size_t)ti.row0 + r;
-        const size_t o = prow * p.d + ti.col0;
-        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-          const int n_left = ti.n_valid - c * 32;
-          if (n_left <= 0) break;
-          uint32_t ra[32];
-          ptx::tmem_ld32(t_row + c * 32, ra);
-          ptx::tmem_ld_wait();
-          float v[32];
+        for (int blk = 0; blk < 2; ++blk) {          // two 64-column blocks per warp
+          const int cb = half * 128 + blk * 64;
+          if (ti.n_valid - cb <= 0) break;
+          stage_open();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
-          store_row32_bf16(p.out_b0 + o + c * 32, v, n_left);
+          for (int cc = 0; cc < 2; ++cc) {
+            uint32_t ra[32];
+            ptx::tmem_ld32(t_row + cb + cc * 32, ra);
+            ptx::tmem_ld_wait();
+            float v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
+            stage_put_bf16(cc * 4, v);
+          }
+          stage_send_2d(&tmC0, ti.col0 + cb, y0);
         }
       } else if (MODE == MODE_DH) {
         const size_t prow = (size_t)ti.row0 + r;
         const float g = gate_of_row(p, (int)prow);
         const size_t gi = prow * p.F + ti.col0;
-        const size_t oi = prow * 2 * (size_t)p.F + ti.col0;
         float dgate = 0.f;
-        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-          const int n_left = ti.n_valid - c * 32;
-          if (n_left <= 0) break;
-          // saved pre-activations of this chunk: issue the loads before waiting on TMEM
-          uint4 g4[4], u4[4];
+        for (int blk = 0; blk < 2; ++blk) {
+          const int cb = half * 128 + blk * 64;
+          if (ti.n_valid - cb <= 0) break;
+          uint32_t pdg[32], pdu[32];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (q * 8 < n_left) {
-              g4[q] = *reinterpret_cast<const uint4*>(p.in_G + gi + c * 32 + q * 8);
-              u4[q] = *reinterpret_cast<const uint4*>(p.in_U + gi + c * 32 + q * 8);
+          for (int cc = 0; cc < 2; ++cc) {
+            const int c0 = cb + cc * 32;
+            const int n_left = ti.n_valid - c0;
+            // saved pre-activations of this chunk: issue the loads before waiting on TMEM
+            uint4 g4[4], u4[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              if (q * 8 < n_left) {
+                g4[q] = *reinterpret_cast<const uint4*>(p.in_G + gi + c0 + q * 8);
+                u4[q] = *reinterpret_cast<const uint4*>(p.in_U + gi + c0 + q * 8);
+              } else {
+                g4[q] = make_uint4(0u, 0u, 0u, 0u);
+                u4[q] = make_uint4(0u, 0u, 0u, 0u);
+              }
             }
-          }
-          uint32_t ra[32];
-          ptx::tmem_ld32(t_row + c * 32, ra);
-          ptx::tmem_ld_wait();
-          float vdg[32], vdu[32];
+            uint32_t ra[32];
+            ptx::tmem_ld32(t_row + c0, ra);
+            ptx::tmem_ld_wait();
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (q * 8 < n_left) {
-              float fg[8], fu[8];
+            for (int q = 0; q < 4; ++q) {
+              float fg[8], fu[8], vdg[8], vdu[8];
               unpack8(g4[q], fg);
               unpack8(u4[q], fu);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
-                const float dA = __uint_as_float(ra[q * 8 + i]);
+                const float dA = (q * 8 < n_left) ? __uint_as_float(ra[q * 8 + i]) : 0.f;
                 const float sg = __fdividef(1.f, 1.f + __expf(-fg[i]));
                 const float si = fg[i] * sg;            // silu(G)
                 dgate += dA * si * fu[i];                // <dA, H>
                 const float dH = g * dA;
-                vdg[q * 8 + i] = dH * fu[i] * sg * (1.f + fg[i] * (1.f - sg));
-                vdu[q * 8 + i] = dH * si;
+                vdg[i] = dH * fu[i] * sg * (1.f + fg[i] * (1.f - sg));
+                vdu[i] = dH * si;
               }
-            } else {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) vdg[q * 8 + i] = vdu[q * 8 + i] = 0.f;
+              for (int i = 0; i < 4; ++i) {
+                pdg[cc * 16 + q * 4 + i] = pack_bf16(vdg[2 * i], vdg[2 * i + 1]);
+                pdu[cc * 16 + q * 4 + i] = pack_bf16(vdu[2 * i], vdu[2 * i + 1]);
+              }
             }
           }
-          store_row32_bf16(p.out_b0 + oi + c * 32, vdg, n_left);
-          store_row32_bf16(p.out_b0 + oi + p.F + c * 32, vdu, n_left);
+          stage_open();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) stage_put(q, pdg[q * 4], pdg[q * 4 + 1], pdg[q * 4 + 2], pdg[q * 4 + 3]);
+          stage_send_2d(&tmC0, ti.col0 + cb, y0);   // dG: columns [0,F) of [dG|dU]
+          stage_open();
+#pragma unroll
+          for (int q = 0; q < 8; ++q) stage_put(q, pdu[q * 4], pdu[q * 4 + 1], pdu[q * 4 + 2], pdu[q * 4 + 3]);
+          stage_send_2d(&tmC1, ti.col0 + cb, y0);   // dU: columns [F,2F)
         }
         const int nt = ti.col0 / BN;
         p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + prow] = dgate;
-      } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile store
-        float* C = p.out_f;
-        size_t ld;
-        if (MODE == MODE_DENSE) {
-          ld = (size_t)p.N;
-        } else {
-          ld = (size_t)p.N;
-          C += (size_t)ti.e * p.M * p.N;
-        }
-        const bool row_ok = r < ti.m_valid;
-        float* crow = C + ((size_t)ti.row0 + r) * ld + ti.col0;
-        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-          const int n_left = ti.n_valid - c * 32;
-          if (n_left <= 0) break;
-          uint32_t ra[32];
-          if (have_acc) {
-            ptx::tmem_ld32(t_row + c * 32, ra);
-            ptx::tmem_ld_wait();
-          } else {
+      } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile, four 32-column blocks per warp
+        if (y0 < ti.row0 + ti.m_valid) {
+          for (int blk = 0; blk < 4; ++blk) {
+            const int cb = half * 128 + blk * 32;
+            if (ti.n_valid - cb <= 0) break;
+            uint32_t ra[32];
+            if (have_acc) {
+              ptx::tmem_ld32(t_row + cb, ra);
+              ptx::tmem_ld_wait();
+            } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) ra[i] = 0u;
-          }
-          if (row_ok) {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              if (q * 4 < n_left) {
-                const uint4 v = make_uint4(ra[q * 4], ra[q * 4 + 1], ra[q * 4 + 2], ra[q * 4 + 3]);
-                *reinterpret_cast<uint4*>(crow + c * 32 + q * 4) = v;
-              }
+              for (int i = 0; i < 32; ++i) ra[i] = 0u;
             }
+            stage_open();
+#pragma unroll
+            for (int q = 0; q < 8; ++q) stage_put(q, ra[q * 4], ra[q * 4 + 1], ra[q * 4 + 2], ra[q * 4 + 3]);
+            stage_send_3d(&tmC0, ti.col0 + cb, y0, ti.e);
           }
         }
       }
@@ -450,6 +491,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         acc_ph ^= 1u;
       }
     }
+    if (lane == 0) ptx::bulk_wait0();   // every tile store of this warp has landed
+    __syncwarp();
   }
 
   // ---- teardown ----
@@ -486,12 +529,14 @@ static EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows, cols] row-major; box = {64 columns, box_rows rows}, 128-byte swizzle, zero fill out of bounds.
-static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// bf16 matrix [rows, cols] with a row pitch of pitch_elems elements; box = {64 columns, box_rows rows},
+// 128-byte swizzle, zero fill (loads) / clipping (stores) out of bounds.
+static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint64_t pitch_elems = 0) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  if (pitch_elems == 0) pitch_elems = cols;
   cuuint64_t gdim[2] = {cols, rows};
-  cuuint64_t gstr[1] = {cols * 2};
+  cuuint64_t gstr[1] = {pitch_elems * 2};
   cuuint32_t box[2] = {64, box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -499,8 +544,25 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t 
   return r == CUDA_SUCCESS;
 }
 
+// fp32 tensor [batch, rows, cols]; box = {32 columns, 32 rows, 1}: the epilogue's store block.
+static bool make_map_f32_out(CUtensorMap* tm, const void* base, uint64_t batch, uint64_t rows, uint64_t cols) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t gdim[3] = {cols, rows, batch};
+  cuuint64_t gstr[2] = {cols * 4, rows * cols * 4};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+struct Maps {
+  CUtensorMap A, B, C0, C1, C2;
+};
+
 template <int MODE, bool A_MN, bool B_MN>
-static cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int grid, cudaStream_t st) {
+static cudaError_t launch_t(const Maps& m, const GemmParams& p, int grid, cudaStream_t st) {
   static bool configured = false;
   auto kern = grouped_gemm_kernel<MODE, A_MN, B_MN>;
   if (!configured) {
@@ -508,7 +570,7 @@ static cudaError_t launch_t(const CUtensorMap& tmA, const CUtensorMap& tmB, cons
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(tmA, tmB, p);
+  kern<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(m.A, m.B, m.C0, m.C1, m.C2, p);
   return cudaGetLastError();
 }
 
@@ -531,48 +593,53 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.gates = gates;
   p.gate_is_f32 = dm.gate_dtype == GROUTER_GATE_F32;
   p.status = ctx->pp.status;
-  CUtensorMap tmA, tmB;
+  Maps m;
   bool ok = true;
   const int grid = ctx->num_sms;
   switch (mode) {
     case MODE_UP:
-      ok = make_map(&tmA, ws.Xp, Rp, d, 128) && make_map(&tmB, W_gu, (uint64_t)E * 2 * F, d, 128);
+      ok = make_map(&m.A, ws.Xp, Rp, d, 128) && make_map(&m.B, W_gu, (uint64_t)E * 2 * F, d, 128) && make_map(&m.C0, ws.G, Rp, F, 32) &&
+           make_map(&m.C1, ws.U, Rp, F, 32) && make_map(&m.C2, ws.Hs, Rp, F, 32);
       p.tiles_n = cdiv(F, 128);
-      p.out_b0 = ws.G; p.out_b1 = ws.U; p.out_b2 = ws.Hs;
       if (!ok) return cudaErrorInvalidValue;
-      return launch_t<MODE_UP, false, false>(tmA, tmB, p, grid, st);
+      return launch_t<MODE_UP, false, false>(m, p, grid, st);
     case MODE_DOWN:
-      ok = make_map(&tmA, ws.Hs, Rp, F, 128) && make_map(&tmB, W_d, (uint64_t)E * d, F, 128);
+      ok = make_map(&m.A, ws.Hs, Rp, F, 128) && make_map(&m.B, W_d, (uint64_t)E * d, F, 128) && make_map(&m.C0, ws.O, Rp, d, 32);
+      m.C1 = m.C2 = m.C0;
       p.tiles_n = cdiv(d, BN);
-      p.out_b0 = ws.O;
       if (!ok) return cudaErrorInvalidValue;
-      return launch_t<MODE_DOWN, false, false>(tmA, tmB, p, grid, st);
+      return launch_t<MODE_DOWN, false, false>(m, p, grid, st);
     case MODE_DH:
-      ok = make_map(&tmA, ws.dYp, Rp, d, 128) && make_map(&tmB, W_d, (uint64_t)E * d, F, 64);
+      // [dG|dU] is one [R_pad, 2F] buffer; the stores see it as two [R_pad, F] views so that clipping stops at F
+      ok = make_map(&m.A, ws.dYp, Rp, d, 128) && make_map(&m.B, W_d, (uint64_t)E * d, F, 64) &&
+           make_map(&m.C0, ws.dGU, Rp, F, 32, 2 * (uint64_t)F) && make_map(&m.C1, ws.dGU + F, Rp, F, 32, 2 * (uint64_t)F);
+      m.C2 = m.C0;
       p.tiles_n = cdiv(F, BN);
-      p.out_b0 = ws.dGU; p.in_G = ws.G; p.in_U = ws.U; p.out_f = ws.dgate_part;
+      p.in_G = ws.G; p.in_U = ws.U; p.out_f = ws.dgate_part;
       if (!ok) return cudaErrorInvalidValue;
-      return launch_t<MODE_DH, false, true>(tmA, tmB, p, grid, st);
+      return launch_t<MODE_DH, false, true>(m, p, grid, st);
     case MODE_DX:
-      ok = make_map(&tmA, ws.dGU, Rp, 2 * (uint64_t)F, 128) && make_map(&tmB, W_gu, (uint64_t)E * 2 * F, d, 64);
+      ok = make_map(&m.A, ws.dGU, Rp, 2 * (uint64_t)F, 128) && make_map(&m.B, W_gu, (uint64_t)E * 2 * F, d, 64) &&
+           make_map(&m.C0, ws.O, Rp, d, 32);
+      m.C1 = m.C2 = m.C0;
       p.tiles_n = cdiv(d, BN);
-      p.out_b0 = ws.O;
       if (!ok) return cudaErrorInvalidValue;
-      return launch_t<MODE_DX, false, true>(tmA, tmB, p, grid, st);
+      return launch_t<MODE_DX, false, true>(m, p, grid, st);
     case MODE_WGRAD_D:
-      ok = make_map(&tmA, ws.dYp, Rp, d, 64) && make_map(&tmB, ws.Hs, Rp, F, 64);
+      ok = make_map(&m.A, ws.dYp, Rp, d, 64) && make_map(&m.B, ws.Hs, Rp, F, 64) && make_map_f32_out(&m.C0, dW_d, E, d, F);
+      m.C1 = m.C2 = m.C0;
       p.M = d; p.N = F;
       p.tiles_m = cdiv(d, BM); p.tiles_n = cdiv(F, BN);
-      p.out_f = dW_d;
       if (!ok) return cudaErrorInvalidValue;
-      return launch_t<MODE_WGRAD_D, true, true>(tmA, tmB, p, grid, st);
+      return launch_t<MODE_WGRAD_D, true, true>(m, p, grid, st);
     case MODE_WGRAD_GU:
-      ok = make_map(&tmA, ws.dGU, Rp, 2 * (uint64_t)F, 64) && make_map(&tmB, ws.Xp, Rp, d, 64);
+      ok = make_map(&m.A, ws.dGU, Rp, 2 * (uint64_t)F, 64) && make_map(&m.B, ws.Xp, Rp, d, 64) &&
+           make_map_f32_out(&m.C0, dW_gu, E, 2 * (uint64_t)F, d);
+      m.C1 = m.C2 = m.C0;
       p.M = 2 * F; p.N = d;
       p.tiles_m = cdiv(2 * F, BM); p.tiles_n = cdiv(d, BN);
-      p.out_f = dW_gu;
       if (!ok) return cudaErrorInvalidValue;
-      return launch_t<MODE_WGRAD_GU, true, true>(tmA, tmB, p, grid, st);
+      return launch_t<MODE_WGRAD_GU, true, true>(m, p, grid, st);
     default:
       return cudaErrorInvalidValue;
   }
@@ -584,21 +651,21 @@ cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, 
   p.M = M; p.N = N; p.K = K;
   p.tiles_m = cdiv(M, BM);
   p.tiles_n = cdiv(N, BN);
-  p.out_f = C;
   p.status = status;
-  CUtensorMap tmA, tmB;
-  const bool ok = (a_mn ? make_map(&tmA, A, K, M, 64) : make_map(&tmA, A, M, K, 128)) &&
-                  (b_mn ? make_map(&tmB, B, K, N, 64) : make_map(&tmB, B, N, K, 128));
+  Maps m;
+  const bool ok = (a_mn ? make_map(&m.A, A, K, M, 64) : make_map(&m.A, A, M, K, 128)) &&
+                  (b_mn ? make_map(&m.B, B, K, N, 64) : make_map(&m.B, B, N, K, 128)) && make_map_f32_out(&m.C0, C, 1, M, N);
   if (!ok) return cudaErrorInvalidValue;
+  m.C1 = m.C2 = m.C0;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   int grid = p.tiles_m * p.tiles_n;
   if (grid > sms) grid = sms;
-  if (a_mn && b_mn) return launch_t<MODE_DENSE, true, true>(tmA, tmB, p, grid, st);
-  if (a_mn) return launch_t<MODE_DENSE, true, false>(tmA, tmB, p, grid, st);
-  if (b_mn) return launch_t<MODE_DENSE, false, true>(tmA, tmB, p, grid, st);
-  return launch_t<MODE_DENSE, false, false>(tmA, tmB, p, grid, st);
+  if (a_mn && b_mn) return launch_t<MODE_DENSE, true, true>(m, p, grid, st);
+  if (a_mn) return launch_t<MODE_DENSE, true, false>(m, p, grid, st);
+  if (b_mn) return launch_t<MODE_DENSE, false, true>(m, p, grid, st);
+  return launch_t<MODE_DENSE, false, false>(m, p, grid, st);
 }
 
 }  // namespace grouter
