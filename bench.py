@@ -32,6 +32,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 from paper_2603_06626_b200 import synth  # noqa: E402
+from paper_2603_06626_b200 import shard  # noqa: E402
 
 METRIC = "moe_layer_fwd_bwd_tokens_per_sec"
 UNIT = "tokens/s"
@@ -65,8 +66,9 @@ def kernel_work(w: synth.Workload):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    """Samples SM clock and throttle reasons with nvidia-smi.  Started before the warm-up (nvidia-smi takes a
+    while to come up); only samples whose timestamp falls inside the timed region are kept."""
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
@@ -75,16 +77,18 @@ class ClockSampler:
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                                           "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin: float, t_end: float):
+        """t_begin/t_end: time.time() at the two ends of the timed region."""
+        import datetime
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
-        time.sleep(0.15)
+        time.sleep(0.1)
         self.proc.terminate()
         try:
             text, _ = self.proc.communicate(timeout=5)
@@ -96,13 +100,16 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in text.strip().splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if ts < t_begin or ts > t_end + 0.05:
+                    continue
+                sm.append(float(parts[1])); mx.append(float(parts[2])); pw.append(float(parts[3]))
             except ValueError:
                 continue
-            for n, v in zip(names, parts[3:7]):
+            for n, v in zip(names, parts[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         if sm:
@@ -145,7 +152,7 @@ def oracle_sample_tokens_per_sec(w: synth.Workload, li, n_tokens: int):
 
 def run_reference(args):
     """Reference arm: the CPU oracle timed on the host cores, same metric and workload config."""
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = shard.env_rank_world()
     if rank != 0:
         return
     w = synth.WORKLOADS[args.workload]
@@ -182,7 +189,7 @@ def workload_config(w: synth.Workload, n_gpus: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="large", choices=list(synth.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
@@ -201,9 +208,7 @@ def main():
     import torch.distributed as dist
     from paper_2603_06626_b200 import binding
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local_rank, world = shard.env_rank_world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
@@ -213,7 +218,7 @@ def main():
     warm = max(args.warmup, 3)
 
     base = synth.WORKLOADS[args.workload]
-    w = synth.reseeded(base, base.seed + 1000 * rank) if rank else base
+    w = shard.rank_workload(base, rank)
     li = synth.make_layer_inputs(w, threads=min(16, os.cpu_count() or 1))
 
     def bf16(a):
@@ -238,36 +243,34 @@ def main():
         layer.backward(dY, X, gates, W_gu, W_d, dX, dW_gu, dW_d, dgates)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        shard.barrier(world)
 
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
     for _ in range(warm):
         step()
     layer.check_status()
     barrier()
     torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     layer.timing_enable(12 * args.steps)
+    wall0 = time.time()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for _ in range(args.steps):
         step()
     ev1.record()
     torch.cuda.synchronize()
+    wall1 = time.time()
     barrier()
     ms_total = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
     per_kernel = layer.timing_read()
     layer.timing_enable(0)
     layer.check_status()
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = shard.max_over_ranks(ms_total, dev, world)
     ms_step = ms_total / args.steps
-    value = world * w.T / (ms_step * 1e-3)
+    value = shard.job_tokens_per_sec(world, w.T, ms_step)
 
     # ---- end to end: host buffers in, host results out, every step ----
     e2e = None
@@ -295,14 +298,11 @@ def main():
         torch.cuda.synchronize()
         barrier()
         ms_e2e = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = shard.max_over_ranks(ms_e2e, dev, world)
         layer.check_status()
         h2d = idx_h.numel() * idx_h.element_size() + gates_h.numel() * 2 + X_h.numel() * 2 + dY_h.numel() * 2
         d2h = Y_h.numel() * 2 + dX_h.numel() * 2 + dg_h.numel() * 4
-        e2e = {"value": world * w.T / (ms_e2e / args.e2e_steps * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": shard.job_tokens_per_sec(world, w.T, ms_e2e / args.e2e_steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": args.e2e_steps,
                "note": "idx, gates, X, dY copied from pinned host memory and Y, dX, dgates copied back every step "
                        "(grouter_moe_step_host); weights and weight gradients stay on the device"}
