@@ -102,6 +102,35 @@ size_t grouter_host_staging_bytes(const grouter_dims* dims);
 int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
                  int32_t* row_to_slot, int32_t* slot_to_row, void* stream);
 
+/* Routing-plan build for callers that cannot allocate device memory (the paper has
+ * no counterpart: this is a deployment aid).  grouter_plan needs a context, and
+ * grouter_create takes its scratch from cudaMalloc.  A host that has given the
+ * whole device to a pooling allocator, runs under a fixed memory budget, or
+ * cannot afford the device-wide synchronisation of an allocation inside its loop
+ * calls this instead: the scratch is a fixed array inside the library image
+ * (about 4.6 MB, present on every GPU that loads the library until the process
+ * exits), and the call makes no cudaMalloc/cudaFree and uses no allocating
+ * library routine.
+ *   Same definition and outputs as grouter_plan (counts, offsets, row_to_slot,
+ *   slot_to_row; bit-identical results); sizes are passed directly.
+ *   idx_dtype: GROUTER_IDX_U8 or GROUTER_IDX_I32.  fold_map: [E_src] or NULL (then E_src == E_tgt).
+ *   status: optional device int32 the kernels OR status bits into (1 = an id or fold
+ *           target was out of range and was treated as expert 0); cleared by the call.
+ *           NULL keeps the word inside the library's scratch, where the caller cannot read it.
+ * Limits: T*k <= 524288 and E_tgt <= 256; larger problems return
+ * GROUTER_ERR_UNSUPPORTED ("unsupported size or type") and must use
+ * grouter_create + grouter_plan.  Other errors as grouter_plan.
+ * The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call outside
+ * any stream capture.  All calls on a device share the one array and it keeps the
+ * previous call's contents (the call clears the words that must start at zero), so
+ * two calls whose kernels may overlap on the GPU (different streams, no ordering
+ * between them) race: order them on one stream or with events.  Nothing from this
+ * call feeds grouter_moe_fwd/bwd, which read the plan kept by a context. */
+int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const int32_t* fold_map, int32_t T, int32_t k, int32_t E_src,
+                         int32_t E_tgt, int32_t* counts, int32_t* offsets, int32_t* row_to_slot, int32_t* slot_to_row,
+                         int32_t* status, void* stream);
+
 /* Forward, Eq. 1:  Y[t,:] = sum_j gates[t,j] * f_{e(t,j)}(X[t,:]).
  *   X     [T,d] bf16             gates [T,k] bf16 or f32 (dims.gate_dtype), used as given
  *   W_gu  [E_tgt, 2*ffn, d] bf16: rows 0..ffn-1 gate projection, ffn..2ffn-1 up projection

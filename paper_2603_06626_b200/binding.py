@@ -19,7 +19,7 @@ GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
-           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read"]
+           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX"]
 
@@ -58,6 +58,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_host_staging_bytes.restype = ctypes.c_size_t
     lib.grouter_plan.argtypes = [vp, vp, i32p, i32p, i32p, i32p, i32p, vp]
     lib.grouter_plan.restype = ctypes.c_int
+    lib.grouter_plan_noalloc.argtypes = [vp, ctypes.c_int32, i32p] + [ctypes.c_int32] * 4 + [i32p] * 5 + [vp]
+    lib.grouter_plan_noalloc.restype = ctypes.c_int
     lib.grouter_moe_fwd.argtypes = [vp] * 8
     lib.grouter_moe_fwd.restype = ctypes.c_int
     lib.grouter_moe_bwd.argtypes = [vp] * 12
@@ -185,6 +187,28 @@ class GrouterLayer:
 
     def check_status(self) -> None:
         _check(self.status(), "device status")
+
+
+def plan_noalloc(idx: torch.Tensor, fold_map: Optional[torch.Tensor], E_src: int, E_tgt: int, out=None, status=None):
+    """Routing plan without a context and without any device allocation inside the library (grouter_plan_noalloc).
+
+    For hosts that may not allocate: pass `out` = (counts[E_tgt], offsets[E_tgt+1], row_to_slot[R], slot_to_row[R])
+    int32 device tensors and an int32[1] `status` tensor you already own, and nothing is allocated anywhere.
+    When they are omitted this wrapper creates them with torch for convenience (the library still allocates nothing).
+    Limits: T*k <= 524288, E_tgt <= 256.  Calls share one scratch array per GPU: keep them ordered on one stream.
+    Returns (counts, offsets, row_to_slot, slot_to_row, status)."""
+    lib = load_library()
+    T, k = idx.shape
+    dt = IDX_U8 if idx.dtype == torch.uint8 else IDX_I32
+    i32 = dict(dtype=torch.int32, device=idx.device)
+    if out is None:
+        out = (torch.empty(E_tgt, **i32), torch.empty(E_tgt + 1, **i32), torch.empty(T * k, **i32), torch.empty(T * k, **i32))
+    if status is None:
+        status = torch.empty(1, **i32)
+    with torch.cuda.device(idx.device):
+        _check(lib.grouter_plan_noalloc(_ptr(idx), dt, _ptr(fold_map), T, k, E_src, E_tgt, _ptr(out[0]), _ptr(out[1]), _ptr(out[2]),
+                                        _ptr(out[3]), _ptr(status), _stream()), "grouter_plan_noalloc")
+    return (*out, status)
 
 
 def dense_gemm(A: torch.Tensor, a_mn_major: bool, B: torch.Tensor, b_mn_major: bool, M: int, N: int, K: int) -> torch.Tensor:

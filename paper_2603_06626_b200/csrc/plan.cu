@@ -241,3 +241,116 @@ cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int3
 }
 
 }  // namespace grouter
+
+// ------------------------------------------------------------------------
+// grouter_plan_noalloc: the same two plan kernels, run without a context.
+//
+// grouter_create owns the plan's scratch (per-block histograms, the ticket of
+// the last-block scan, the padded copy of the permutation) in memory it gets
+// from cudaMalloc.  Some hosts cannot make that call: a process that has
+// handed the whole device to a pooling allocator with a fixed reservation, a
+// plug-in running under a memory budget it may not exceed, or a
+// latency-critical loop that cannot take the device-wide synchronisation an
+// allocation implies.  For them the scratch lives in the library image itself:
+// one file-scope __device__ array that every GPU loading the library holds
+// until the process exits.  Its size fixes the largest problem this entry
+// point accepts.
+// ------------------------------------------------------------------------
+namespace grouter {
+namespace {
+
+constexpr int NOALLOC_MAX_R = 1 << 19;       // routed slots T*k
+constexpr int NOALLOC_MAX_E = 256;           // target experts
+constexpr int NOALLOC_MAX_ROWS = NOALLOC_MAX_R + ROW_TILE * NOALLOC_MAX_E;          // padded rows
+constexpr int NOALLOC_MAX_BLOCKS = NOALLOC_MAX_R / PLAN_MIN_CHUNK;                   // plan_geom never uses more
+// layout of the scratch, in 32-bit words (every part starts on a 256-byte boundary)
+constexpr int NA_PAD_OFFSETS = 0;                                     // [E+1]
+constexpr int NA_ROW_SHIFT = NA_PAD_OFFSETS + 320;                    // [E]
+constexpr int NA_PAD_BEGIN = NA_ROW_SHIFT + 256;                      // [E]
+constexpr int NA_N_TILES = NA_PAD_BEGIN + 256;                        // [1]
+constexpr int NA_TICKET = NA_N_TILES + 64;                            // [1]
+constexpr int NA_STATUS = NA_TICKET + 64;                             // [1] used when the caller passes no status word
+constexpr int NA_TILE_EXPERT = NA_STATUS + 64;                        // [rows/128]
+constexpr int NA_SLOT_TO_PROW = NA_TILE_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE;   // [R]
+constexpr int NA_PROW_TO_SLOT = NA_SLOT_TO_PROW + NOALLOC_MAX_R;      // [rows]
+constexpr int NA_BLK_PREFIX = NA_PROW_TO_SLOT + NOALLOC_MAX_ROWS;     // [E * blocks]
+constexpr int NA_WORDS = NA_BLK_PREFIX + NOALLOC_MAX_E * NOALLOC_MAX_BLOCKS;
+static_assert(NA_TILE_EXPERT % 64 == 0 && NA_SLOT_TO_PROW % 64 == 0 && NA_PROW_TO_SLOT % 64 == 0 && NA_BLK_PREFIX % 64 == 0,
+              "scratch parts must start on 256-byte boundaries");
+
+// About 4.6 MB per GPU.  In host code this name is only a handle for cudaGetSymbolAddress: it is not a
+// device address and must never be handed to a kernel as one.
+static __device__ __align__(256) int32_t g_plan_scratch[NA_WORDS];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+int32_t* g_plan_scratch_addr[NOALLOC_MAX_DEVICES] = {};   // device address of the array, per device, once looked up
+
+// Device address of this device's copy of the scratch array (looked up on the first call per device).
+int32_t* plan_scratch_on_current_device(int* rc) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) {
+    *rc = GROUTER_ERR_NO_DEVICE;
+    return nullptr;
+  }
+  int32_t* p = __atomic_load_n(&g_plan_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (p == nullptr) {
+    void* sym = nullptr;
+    if (cudaGetSymbolAddress(&sym, g_plan_scratch) != cudaSuccess || sym == nullptr) {
+      *rc = GROUTER_ERR_CUDA;
+      return nullptr;
+    }
+    p = static_cast<int32_t*>(sym);
+    __atomic_store_n(&g_plan_scratch_addr[dev], p, __ATOMIC_RELEASE);   // racing threads store the same value
+  }
+  *rc = GROUTER_OK;
+  return p;
+}
+
+}  // namespace
+}  // namespace grouter
+
+extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const int32_t* fold_map, int32_t T, int32_t k, int32_t E_src,
+                                    int32_t E_tgt, int32_t* counts, int32_t* offsets, int32_t* row_to_slot, int32_t* slot_to_row,
+                                    int32_t* status, void* stream) {
+  using namespace grouter;
+  if (!idx || !counts || !offsets || !row_to_slot || !slot_to_row) return GROUTER_ERR_INVALID_ARG;
+  if (T < 1 || k < 1 || E_src < 1 || E_tgt < 1) return GROUTER_ERR_INVALID_ARG;
+  if (idx_dtype != GROUTER_IDX_U8 && idx_dtype != GROUTER_IDX_I32) return GROUTER_ERR_INVALID_ARG;
+  if (!fold_map && E_src != E_tgt) return GROUTER_ERR_INVALID_ARG;
+  if (idx_dtype == GROUTER_IDX_U8 && E_src > 256) return GROUTER_ERR_UNSUPPORTED;
+  // beyond the fixed scratch: the caller has to use grouter_create + grouter_plan
+  if ((int64_t)T * k > NOALLOC_MAX_R || E_tgt > NOALLOC_MAX_E) return GROUTER_ERR_UNSUPPORTED;
+  auto misaligned = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (misaligned(idx) || misaligned(counts) || misaligned(offsets) || misaligned(row_to_slot) || misaligned(slot_to_row) ||
+      (fold_map && misaligned(fold_map)) || (status && (reinterpret_cast<uintptr_t>(status) & 3u)))
+    return GROUTER_ERR_MISALIGNED;
+  int rc = GROUTER_OK;
+  int32_t* base = plan_scratch_on_current_device(&rc);
+  if (!base) return rc;
+
+  grouter_ctx c{};   // lives on the host stack for the duration of the two launches
+  c.dims.T = T; c.dims.d = 8; c.dims.ffn = 8; c.dims.E_src = E_src; c.dims.E_tgt = E_tgt; c.dims.k = k;
+  c.dims.idx_dtype = idx_dtype; c.dims.gate_dtype = GROUTER_GATE_BF16;
+  c.R = (int64_t)T * k;
+  c.geom = plan_geom(c.R);
+  c.pp.pad_offsets = base + NA_PAD_OFFSETS;
+  c.pp.row_shift = base + NA_ROW_SHIFT;
+  c.pp.pad_begin = base + NA_PAD_BEGIN;
+  c.pp.n_m_tiles = base + NA_N_TILES;
+  c.pp.ticket = reinterpret_cast<unsigned int*>(base + NA_TICKET);
+  c.pp.status = status ? status : base + NA_STATUS;
+  c.pp.tile_expert = base + NA_TILE_EXPERT;
+  c.pp.slot_to_prow = base + NA_SLOT_TO_PROW;
+  c.pp.prow_to_slot = base + NA_PROW_TO_SLOT;
+  c.pp.blk_prefix = base + NA_BLK_PREFIX;
+  if (c.geom.nblk > NOALLOC_MAX_BLOCKS) return GROUTER_ERR_UNSUPPORTED;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The array still holds whatever the previous call left.  The ticket must count from zero and the status
+  // word must start clear; every other part is overwritten before it is read.
+  if (cudaMemsetAsync(c.pp.ticket, 0, sizeof(unsigned int), st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemsetAsync(c.pp.status, 0, sizeof(int32_t), st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  for (int phase = 0; phase < 2; ++phase)
+    if (launch_plan(&c, phase, idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  return GROUTER_OK;
+}
