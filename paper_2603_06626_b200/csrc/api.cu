@@ -163,7 +163,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   size_t off = 0;
   auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
   const size_t o_pad = take((size_t)(E + 1) * 4), o_shift = take((size_t)E * 4), o_pb = take((size_t)E * 4);
-  const size_t o_te = take((size_t)c->max_m_tiles * 4), o_nt = take(4), o_s2p = take((size_t)c->R * 4);
+  const size_t o_pr = take((size_t)c->max_m_tiles * 4), o_pe = take((size_t)c->max_m_tiles * 4), o_nt = take(4), o_s2p = take((size_t)c->R * 4);
   const size_t o_p2s = take((size_t)c->R_pad_max * 4), o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
   if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
     delete c;
@@ -178,8 +178,9 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.pad_offsets = reinterpret_cast<int32_t*>(b + o_pad);
   c->pp.row_shift = reinterpret_cast<int32_t*>(b + o_shift);
   c->pp.pad_begin = reinterpret_cast<int32_t*>(b + o_pb);
-  c->pp.tile_expert = reinterpret_cast<int32_t*>(b + o_te);
-  c->pp.n_m_tiles = reinterpret_cast<int32_t*>(b + o_nt);
+  c->pp.pair_row0 = reinterpret_cast<int32_t*>(b + o_pr);
+  c->pp.pair_expert = reinterpret_cast<int32_t*>(b + o_pe);
+  c->pp.n_pair_tiles = reinterpret_cast<int32_t*>(b + o_nt);
   c->pp.slot_to_prow = reinterpret_cast<int32_t*>(b + o_s2p);
   c->pp.prow_to_slot = reinterpret_cast<int32_t*>(b + o_p2s);
   c->pp.blk_prefix = reinterpret_cast<int32_t*>(b + o_bp);

@@ -13,7 +13,8 @@ namespace grouter {
 constexpr int STATUS_BAD_INDEX = 1;
 constexpr int STATUS_TIMEOUT = 2;
 
-constexpr int ROW_TILE = 128;        // rows of one GEMM tile; expert segments are padded to it
+constexpr int ROW_TILE = 128;        // rows one CTA owns in a GEMM tile; expert segments are padded to it
+constexpr int PAIR_VALID2 = 1 << 30; // flag in PaddedPlan::pair_expert
 constexpr int PLAN_THREADS = 256;    // 8 warps per plan block
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
 constexpr int PLAN_MIN_CHUNK = 2048; // slots per plan block (lower bound)
@@ -40,8 +41,11 @@ struct PaddedPlan {
   int32_t* pad_offsets;   // [E_tgt+1] first padded row of each expert; [E_tgt] = rows in use
   int32_t* row_shift;     // [E_tgt]   pad_offsets[e] - offsets[e]
   int32_t* pad_begin;     // [E_tgt]   first pad row of expert e (pad_offsets[e] + counts[e])
-  int32_t* tile_expert;   // [max_m_tiles] expert of each 128-row tile
-  int32_t* n_m_tiles;     // [1]
+  // Tile list of the row-parallel GEMMs.  A tile is 256 rows of one expert (two 128-row halves, one per CTA
+  // of a pair); an expert with an odd number of 128-row blocks ends in a tile whose second half is unused.
+  int32_t* pair_row0;     // [max_m_tiles] first padded row of each 256-row tile
+  int32_t* pair_expert;   // [max_m_tiles] expert of the tile; bit 30 set when the second half holds rows of that expert
+  int32_t* n_pair_tiles;  // [1]
   int32_t* slot_to_prow;  // [R]
   int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows
   int32_t* blk_prefix;    // [E_tgt * nblk] per-block histogram, then exclusive prefix over blocks

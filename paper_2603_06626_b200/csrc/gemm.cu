@@ -9,27 +9,32 @@
 //   WGRAD_GU  dW_gu[e] = [dG|dU]_e^T * Xp_e
 //   DENSE     C = A * B on plain matrices (component check)
 //
-// Tile: 128 x 256 x 64 per CTA, one CTA per SM.  Warp 0 issues TMA tile loads
-// (128-byte swizzle) into a 4-stage shared-memory ring; warp 1 issues
-// tcgen05.mma (M=128, N=256, K=16) into one of two 256-column TMEM
-// accumulators; warps 2-9 drain the other accumulator with tcgen05.ld and run
-// the fused epilogue, so the epilogue of tile i overlaps the main loop of tile
-// i+1.  Operands may be K-major (rows of the stored matrix run along K) or
-// MN-major (rows run along M/N); both are described to the MMA by
-// shared-memory descriptors, so no operand is ever transposed in memory.
+// Tile: 256 x 256 x 64 per CTA pair (a cluster of two CTAs on neighbouring SMs, one pair-wide tcgen05.mma with
+// M = 256).  Each CTA owns 128 rows of the tile and half of B's 256 columns, so per 64-deep k-step it stages
+// 16 KB of A and 16 KB of B: a third less operand traffic per FLOP than a one-CTA 128 x 256 tile and room for a
+// 6-stage ring.  In every CTA warp 0 issues its TMA tile loads (128-byte swizzle; the byte counts of both CTAs
+// complete on the leader CTA's barrier); warp 1 of the leader CTA issues the MMAs for the pair into one of two
+// 256-column TMEM accumulators (present in both CTAs) and releases stages / publishes accumulators to both
+// CTAs with multicast commits; warps 2-9 of each CTA drain the other accumulator with tcgen05.ld and run the
+// fused epilogue on their CTA's 128 rows, so the epilogue of tile i overlaps the main loop of tile i+1.
+// Operands may be K-major (rows of the stored matrix run along K) or MN-major (rows run along M/N); both are
+// described to the MMA by shared-memory descriptors, so no operand is ever transposed in memory.
 //
-// Every mbarrier wait is bounded; on give-up the CTA raises an abort flag, ORs
-// STATUS_TIMEOUT into the status word, leaves its loops, frees TMEM and exits.
+// Every mbarrier wait is bounded; on give-up the CTA raises an abort flag, ORs STATUS_TIMEOUT into the status
+// word, leaves its loops, and the pair meets at a cluster barrier before freeing TMEM and exiting.
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace grouter {
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int STAGES = 4;
+constexpr int BM = 128;                         // rows of the tile owned by one CTA
+constexpr int PM = 2 * BM;                      // rows of the pair's tile
+constexpr int BN = 256, BK = 64;
+constexpr int BNH = BN / 2;                     // B columns staged by one CTA
+constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;            // 16 KB
-constexpr int B_BYTES = BN * BK * 2;            // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 48 KB
+constexpr int B_BYTES = BNH * BK * 2;           // 16 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 32 KB per CTA and stage
 constexpr int ATOM_BYTES = 64 * BK * 2;         // one 64x64 bf16 box = 8 KB
 constexpr int EPI_WARPS = 8;                    // two warps per TMEM lane quadrant, each takes half of the columns
 constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;
@@ -39,8 +44,9 @@ constexpr uint32_t TMEM_COLS = 512;
 
 struct GemmParams {
   // schedule
-  const int32_t* n_m_tiles;    // device scalar: 128-row tiles in use (row-parallel modes)
-  const int32_t* tile_expert;  // device [tiles]
+  const int32_t* n_pair_tiles; // device scalar: 256-row tiles in use (row-parallel modes)
+  const int32_t* pair_row0;    // device [tiles] first padded row
+  const int32_t* pair_expert;  // device [tiles] expert | PAIR_VALID2
   const int32_t* pad_offsets;  // device [E+1]
   int32_t E, d, F;
   int32_t M, N, K;             // DENSE: problem; WGRAD: per-expert output M x N
@@ -56,59 +62,57 @@ struct GemmParams {
   int32_t* status;
 };
 
-struct Tile {
-  int a_x, a_y;   // TMA coordinates of the A tile at k-step 0
-  int b_x, b_y, b_y2;
+struct Tile {     // one CTA's share of a pair tile
+  int a_x, a_y;   // TMA coordinates of this CTA's A rows at k-step 0
+  int b_x, b_y;   // ... and of this CTA's half of B
   int num_k;
-  int row0, col0; // output origin (row within the output matrix of this problem)
+  int row0, col0; // origin of this CTA's 128 x 256 output block within the output matrix of this problem
   int e;
-  int m_valid, n_valid;
+  int m_valid, n_valid;   // m_valid <= 0: this CTA's rows are not part of the problem (it still feeds its B half)
 };
 
 template <int MODE>
 __device__ __forceinline__ int total_tiles(const GemmParams& p) {
   if (MODE == MODE_WGRAD_D || MODE == MODE_WGRAD_GU) return p.E * p.tiles_m * p.tiles_n;
   if (MODE == MODE_DENSE) return p.tiles_m * p.tiles_n;
-  return __ldg(p.n_m_tiles) * p.tiles_n;
+  return __ldg(p.n_pair_tiles) * p.tiles_n;
 }
 
+// Share of pair tile t that CTA `rank` (0 = leader) of the pair works on.
 template <int MODE>
-__device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t) {
+__device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank) {
   Tile ti;
   if (MODE == MODE_UP || MODE == MODE_DOWN || MODE == MODE_DH || MODE == MODE_DX) {
     const int mt = t / p.tiles_n, nt = t - mt * p.tiles_n;
-    ti.e = __ldg(p.tile_expert + mt);
-    ti.row0 = mt * BM;
-    ti.m_valid = BM;
+    const int pe = __ldg(p.pair_expert + mt);
+    ti.e = pe & ~PAIR_VALID2;
+    ti.row0 = __ldg(p.pair_row0 + mt) + rank * BM;
+    ti.m_valid = (rank == 0 || (pe & PAIR_VALID2)) ? BM : 0;
     ti.a_x = 0;
     ti.a_y = ti.row0;
-    if (MODE == MODE_UP) {          // B = W_gu as [E*2F, d], K-major; 128 gate rows + 128 up rows
+    if (MODE == MODE_UP) {          // B = W_gu as [E*2F, d], K-major; leader stages 128 gate rows, peer the 128 up rows
       ti.col0 = nt * 128;
       ti.n_valid = min(128, p.F - ti.col0);
       ti.b_x = 0;
-      ti.b_y = ti.e * 2 * p.F + ti.col0;
-      ti.b_y2 = ti.b_y + p.F;
+      ti.b_y = ti.e * 2 * p.F + rank * p.F + ti.col0;
       ti.num_k = (p.d + BK - 1) / BK;
     } else if (MODE == MODE_DOWN) { // B = W_d as [E*d, F], K-major
       ti.col0 = nt * BN;
       ti.n_valid = min(BN, p.d - ti.col0);
       ti.b_x = 0;
-      ti.b_y = ti.e * p.d + ti.col0;
-      ti.b_y2 = ti.b_y + 128;
+      ti.b_y = ti.e * p.d + ti.col0 + rank * BNH;
       ti.num_k = (p.F + BK - 1) / BK;
     } else if (MODE == MODE_DH) {   // B = W_d as [E*d, F], MN-major (N = F contiguous), K = d
       ti.col0 = nt * BN;
       ti.n_valid = min(BN, p.F - ti.col0);
-      ti.b_x = ti.col0;
+      ti.b_x = ti.col0 + rank * BNH;
       ti.b_y = ti.e * p.d;
-      ti.b_y2 = 0;
       ti.num_k = (p.d + BK - 1) / BK;
     } else {                        // DX: B = W_gu as [E*2F, d], MN-major (N = d contiguous), K = 2F
       ti.col0 = nt * BN;
       ti.n_valid = min(BN, p.d - ti.col0);
-      ti.b_x = ti.col0;
+      ti.b_x = ti.col0 + rank * BNH;
       ti.b_y = ti.e * 2 * p.F;
-      ti.b_y2 = 0;
       ti.num_k = (2 * p.F + BK - 1) / BK;
     }
   } else if (MODE == MODE_WGRAD_D || MODE == MODE_WGRAD_GU) {
@@ -117,28 +121,26 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t) {
     const int r = t - ti.e * per;
     const int mt = r / p.tiles_n, nt = r - mt * p.tiles_n;
     const int k0 = __ldg(p.pad_offsets + ti.e), k1 = __ldg(p.pad_offsets + ti.e + 1);
-    ti.row0 = mt * BM;
+    ti.row0 = mt * PM + rank * BM;
     ti.col0 = nt * BN;
     ti.m_valid = min(BM, p.M - ti.row0);
     ti.n_valid = min(BN, p.N - ti.col0);
     ti.a_x = ti.row0;   // both operands MN-major: x runs along M/N, y along the expert's rows
     ti.a_y = k0;
-    ti.b_x = ti.col0;
+    ti.b_x = ti.col0 + rank * BNH;
     ti.b_y = k0;
-    ti.b_y2 = 0;
     ti.num_k = (k1 - k0) / BK;
   } else {  // DENSE
     const int mt = t / p.tiles_n, nt = t - mt * p.tiles_n;
     ti.e = 0;
-    ti.row0 = mt * BM;
+    ti.row0 = mt * PM + rank * BM;
     ti.col0 = nt * BN;
     ti.m_valid = min(BM, p.M - ti.row0);
     ti.n_valid = min(BN, p.N - ti.col0);
-    ti.a_x = ti.row0;  // interpreted per operand major below
+    ti.a_x = ti.row0;                 // MN-major A: x; K-major A: y (set below)
     ti.a_y = ti.row0;
-    ti.b_x = ti.col0;
-    ti.b_y = ti.col0;
-    ti.b_y2 = ti.col0 + 128;
+    ti.b_x = ti.col0 + rank * BNH;    // MN-major B: x; K-major B: y
+    ti.b_y = ti.col0 + rank * BNH;
     ti.num_k = (p.K + BK - 1) / BK;
   }
   return ti;
@@ -166,15 +168,21 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
 }
 
 template <int MODE, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(GEMM_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                     const __grid_constant__ CUtensorMap tmC2, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
+  // The dynamic shared memory starts at the same offset in both CTAs of the pair, so every address derived
+  // below names the same location in either CTA (the MMA descriptors and multicast commits rely on that).
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stage_base = smem_base + STAGES * STAGE_BYTES;          // epilogue staging, 4 KB per warp
   const uint32_t bar_base = stage_base + EPI_WARPS * EPI_STAGE_BYTES;
   // barriers (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+  //   full[s]       leader only: one arrival (leader's producer, with the byte count of BOTH CTAs' loads)
+  //   empty[s]      each CTA: one arrival per round, delivered to both CTAs by the leader's multicast commit
+  //   tmem_full[a]  each CTA: one arrival per tile, delivered to both CTAs by the leader's multicast commit
+  //   tmem_empty[a] leader only: 2 * EPI_WARPS arrivals, one per epilogue warp of either CTA
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
@@ -184,6 +192,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const int rank = (int)ptx::cluster_ctarank();      // 0 = leader of the pair
+  const int pair_id = blockIdx.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
     s_abort = 0;
@@ -193,7 +204,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(tfull_bar(a), 1);
-      ptx::mbar_init(tempty_bar(a), EPI_WARPS);
+      ptx::mbar_init(tempty_bar(a), 2 * EPI_WARPS);
     }
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
@@ -203,11 +214,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (MODE == MODE_UP) ptx::prefetch_tensormap(&tmC2);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&s_tmem_base), TMEM_COLS);
-    ptx::tmem_relinquish();
+    ptx::tmem_alloc_pair(ptx::smem_u32(&s_tmem_base), TMEM_COLS);
+    ptx::tmem_relinquish_pair();
   }
   ptx::tc_fence_before();
   __syncthreads();
+  ptx::cluster_sync_all();      // the peer's barriers are initialised and its TMEM is allocated
   ptx::tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
   volatile int* abort_flag = &s_abort;
@@ -215,32 +227,32 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int n_tiles = total_tiles<MODE>(p);
 
   if (warp == 0) {
-    // ===================== TMA producer =====================
+    // ===================== TMA producer (both CTAs) =====================
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
-      for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
-        const Tile ti = decode_tile<MODE>(p, t);
+      for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
+        const Tile ti = decode_tile<MODE>(p, t, rank);
         for (int ks = 0; ks < ti.num_k; ++ks) {
           if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) break;
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
-          const uint32_t fb = full_bar(s);
-          ptx::mbar_arrive_expect_tx(fb, STAGE_BYTES);
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+          const uint32_t fb = ptx::map_to_cta(full_bar(s), 0);   // both CTAs' bytes complete on the leader's barrier
           const int k0 = ks * BK;
           if (!A_MN) {
-            ptx::tma_load_2d(sa, &tmA, fb, k0, ti.a_y);                       // box {64 k, 128 rows}
+            ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y);                       // box {64 k, 128 rows}
           } else {
-            ptx::tma_load_2d(sa, &tmA, fb, ti.a_x, (MODE == MODE_DENSE ? 0 : ti.a_y) + k0);              // box {64 m, 64 k}
-            ptx::tma_load_2d(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, (MODE == MODE_DENSE ? 0 : ti.a_y) + k0);
+            const int ay = (MODE == MODE_DENSE ? 0 : ti.a_y) + k0;
+            ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay);                       // 2 x box {64 m, 64 k}
+            ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay);
           }
           if (!B_MN) {
-            ptx::tma_load_2d(sb, &tmB, fb, k0, ti.b_y);                       // 2 x box {64 k, 128 rows}
-            ptx::tma_load_2d(sb + B_BYTES / 2, &tmB, fb, k0, ti.b_y2);
+            ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y);                       // box {64 k, 128 rows}
           } else {
             const int by = (MODE == MODE_DENSE ? 0 : ti.b_y) + k0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) ptx::tma_load_2d(sb + i * ATOM_BYTES, &tmB, fb, ti.b_x + 64 * i, by);  // box {64 n, 64 k}
+            ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by);                       // 2 x box {64 n, 64 k}
+            ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by);
           }
           if (++s == STAGES) {
             s = 0;
@@ -248,21 +260,30 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
+      // every stage release the leader has multicast to this CTA must have landed before the CTA may exit
+      for (int i = 0; i < STAGES && !*abort_flag; ++i) {
+        if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) break;
+        if (++s == STAGES) {
+          s = 0;
+          ph ^= 1u;
+        }
+      }
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ===================== MMA issuer =====================
-    if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, A_MN, B_MN);
+    // ===================== MMA issuer (leader CTA only) =====================
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(PM, BN, A_MN, B_MN);
       // K-major: 8-row groups are 1024 B apart (SBO); 16 K-elements = 32 B further along the row.
       // MN-major: 64-wide MN atoms are one 8 KB box apart (LBO), 8-k groups 1024 B apart (SBO);
       //           16 K-elements = 16 rows of 128 B = 2048 B further.
       constexpr uint32_t a_lbo = A_MN ? ATOM_BYTES : 16, a_sbo = 1024, a_kadv = A_MN ? 2048 : 32;
       constexpr uint32_t b_lbo = B_MN ? ATOM_BYTES : 16, b_sbo = 1024, b_kadv = B_MN ? 2048 : 32;
+      constexpr uint16_t both = 3;
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
-      for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
-        const Tile ti = decode_tile<MODE>(p, t);
+      for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
+        const Tile ti = decode_tile<MODE>(p, t, 0);
         if (!ptx::mbar_wait_bounded(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
@@ -279,17 +300,21 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           for (int kk = 0; kk < BK / 16; ++kk) {
             const uint64_t da = ptx::make_smem_desc_sw128(sa + kk * a_kadv, a_lbo, a_sbo);
             const uint64_t db = ptx::make_smem_desc_sw128(sb + kk * b_kadv, b_lbo, b_sbo);
-            ptx::umma_bf16(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
+            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
           }
-          ptx::umma_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+          ptx::umma_commit_pair(empty_bar(s), both);  // stage reusable in both CTAs once these MMAs have read it
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
           }
         }
         if (!ok) break;
-        if (ti.num_k > 0) ptx::umma_commit(tfull_bar(acc));
-        else ptx::mbar_arrive(tfull_bar(acc));
+        if (ti.num_k > 0) {
+          ptx::umma_commit_pair(tfull_bar(acc), both);
+        } else {                                      // nothing to contract: the epilogues write zeros
+          ptx::mbar_arrive(tfull_bar(acc));
+          ptx::mbar_arrive_cluster(ptx::map_to_cta(tfull_bar(acc), 1));
+        }
         if (++acc == 2) {
           acc = 0;
           acc_ph ^= 1u;
@@ -340,17 +365,19 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     };
     int acc = 0;
     uint32_t acc_ph = 0;
-    for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
-      const Tile ti = decode_tile<MODE>(p, t);
+    const uint32_t leader_tempty[2] = {ptx::map_to_cta(tempty_bar(0), 0), ptx::map_to_cta(tempty_bar(1), 0)};
+    for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
+      const Tile ti = decode_tile<MODE>(p, t, rank);
       if (!ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag)) break;
       ptx::tc_fence_after();
       const uint32_t t_row = tmem_base + (uint32_t)acc * BN + ((uint32_t)(quad * 32) << 16);
       const bool have_acc = ti.num_k > 0;
       const int y0 = ti.row0 + quad * 32;  // first output row of this warp's block
 
+      const bool live = ti.m_valid > 0;    // false: this CTA only lent its half of B to the pair
       if (MODE == MODE_UP) {
         // accumulator columns 0..127 = gate, 128..255 = up, for F-columns col0..col0+127; this warp: 64 of them
-        if (ti.n_valid - half * 64 > 0) {
+        if (live && ti.n_valid - half * 64 > 0) {
           const float g = gate_of_row(p, ti.row0 + r);
           uint32_t pg[32], pu[32], ph[32];   // packed bf16 pairs: 64 columns each
 #pragma unroll
@@ -386,7 +413,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       } else if (MODE == MODE_DOWN || MODE == MODE_DX) {
         for (int blk = 0; blk < 2; ++blk) {          // two 64-column blocks per warp
           const int cb = half * 128 + blk * 64;
-          if (ti.n_valid - cb <= 0) break;
+          if (!live || ti.n_valid - cb <= 0) break;
           stage_open();
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
@@ -402,12 +429,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       } else if (MODE == MODE_DH) {
         const size_t prow = (size_t)ti.row0 + r;
-        const float g = gate_of_row(p, (int)prow);
+        const float g = live ? gate_of_row(p, (int)prow) : 0.f;
         const size_t gi = prow * p.F + ti.col0;
         float dgate = 0.f;
         for (int blk = 0; blk < 2; ++blk) {
           const int cb = half * 128 + blk * 64;
-          if (ti.n_valid - cb <= 0) break;
+          if (!live || ti.n_valid - cb <= 0) break;
           uint32_t pdg[32], pdu[32];
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
@@ -460,7 +487,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           stage_send_2d(&tmC1, ti.col0 + cb, y0);   // dU: columns [F,2F)
         }
         const int nt = ti.col0 / BN;
-        p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + prow] = dgate;
+        if (live) p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + prow] = dgate;
       } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile, four 32-column blocks per warp
         if (y0 < ti.row0 + ti.m_valid) {
           for (int blk = 0; blk < 4; ++blk) {
@@ -485,7 +512,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // all TMEM reads of this warp are complete (wait::ld above): hand the accumulator back
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+      if (lane == 0) ptx::mbar_arrive_cluster(leader_tempty[acc]);
       if (++acc == 2) {
         acc = 0;
         acc_ph ^= 1u;
@@ -498,15 +525,16 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // ---- teardown ----
   if (*abort_flag) {
     if (threadIdx.x == 0) atomicOr(p.status, STATUS_TIMEOUT);
-    // give copies still in flight towards this CTA's shared memory time to land
+    // give copies and barrier arrivals still in flight towards either CTA's shared memory time to land
     const uint64_t t0 = ptx::globaltimer_ns();
     while (ptx::globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
   }
   ptx::tc_fence_before();
   __syncthreads();
+  ptx::cluster_sync_all();      // neither CTA leaves while the other may still touch its shared memory or TMEM
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
 }
 
@@ -582,8 +610,9 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   const uint64_t Rp = (uint64_t)ctx->R_pad_max;
   const int d = dm.d, F = dm.ffn, E = dm.E_tgt;
   GemmParams p{};
-  p.n_m_tiles = ctx->pp.n_m_tiles;
-  p.tile_expert = ctx->pp.tile_expert;
+  p.n_pair_tiles = ctx->pp.n_pair_tiles;
+  p.pair_row0 = ctx->pp.pair_row0;
+  p.pair_expert = ctx->pp.pair_expert;
   p.pad_offsets = ctx->pp.pad_offsets;
   p.E = E;
   p.d = d;
@@ -595,7 +624,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.status = ctx->pp.status;
   Maps m;
   bool ok = true;
-  const int grid = ctx->num_sms;
+  const int grid = ctx->num_sms & ~1;   // whole CTA pairs, one CTA per SM
   switch (mode) {
     case MODE_UP:
       ok = make_map(&m.A, ws.Xp, Rp, d, 128) && make_map(&m.B, W_gu, (uint64_t)E * 2 * F, d, 128) && make_map(&m.C0, ws.G, Rp, F, 32) &&
@@ -629,7 +658,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
       ok = make_map(&m.A, ws.dYp, Rp, d, 64) && make_map(&m.B, ws.Hs, Rp, F, 64) && make_map_f32_out(&m.C0, dW_d, E, d, F);
       m.C1 = m.C2 = m.C0;
       p.M = d; p.N = F;
-      p.tiles_m = cdiv(d, BM); p.tiles_n = cdiv(F, BN);
+      p.tiles_m = cdiv(d, PM); p.tiles_n = cdiv(F, BN);
       if (!ok) return cudaErrorInvalidValue;
       return launch_t<MODE_WGRAD_D, true, true>(m, p, grid, st);
     case MODE_WGRAD_GU:
@@ -637,7 +666,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
            make_map_f32_out(&m.C0, dW_gu, E, 2 * (uint64_t)F, d);
       m.C1 = m.C2 = m.C0;
       p.M = 2 * F; p.N = d;
-      p.tiles_m = cdiv(2 * F, BM); p.tiles_n = cdiv(d, BN);
+      p.tiles_m = cdiv(2 * F, PM); p.tiles_n = cdiv(d, BN);
       if (!ok) return cudaErrorInvalidValue;
       return launch_t<MODE_WGRAD_GU, true, true>(m, p, grid, st);
     default:
@@ -649,7 +678,7 @@ cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, 
                               cudaStream_t st) {
   GemmParams p{};
   p.M = M; p.N = N; p.K = K;
-  p.tiles_m = cdiv(M, BM);
+  p.tiles_m = cdiv(M, PM);
   p.tiles_n = cdiv(N, BN);
   p.status = status;
   Maps m;
@@ -660,8 +689,8 @@ cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, 
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  int grid = p.tiles_m * p.tiles_n;
-  if (grid > sms) grid = sms;
+  int grid = 2 * p.tiles_m * p.tiles_n;   // one CTA pair per tile, at most one CTA per SM
+  if (grid > (sms & ~1)) grid = sms & ~1;
   if (a_mn && b_mn) return launch_t<MODE_DENSE, true, true>(m, p, grid, st);
   if (a_mn) return launch_t<MODE_DENSE, true, false>(m, p, grid, st);
   if (b_mn) return launch_t<MODE_DENSE, false, true>(m, p, grid, st);

@@ -60,7 +60,7 @@ template <typename IdxT>
 __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
                                                                  int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
                                                                  int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
-  extern __shared__ int32_t sm[];  // max(PLAN_WARPS*E, 3*E+3) ints
+  extern __shared__ int32_t sm[];  // max(PLAN_WARPS*E, 4*E+4) ints
   __shared__ int s_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   int32_t* s_cnt = sm;                    // [E]
   int32_t* s_off = sm + E_tgt;            // [E+1]
   int32_t* s_pad = sm + 2 * E_tgt + 1;    // [E+1]
+  int32_t* s_pair = sm + 3 * E_tgt + 2;   // [E+1] exclusive prefix of 256-row tiles per expert
   __syncthreads();
   for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
     int carry = 0;
@@ -108,31 +109,39 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   if (warp == 0) {
     const int per = (E_tgt + 31) / 32;
     const int e0 = min(lane * per, E_tgt), e1 = min(e0 + per, E_tgt);
-    int sum = 0, psum = 0;
+    int sum = 0, psum = 0, tsum = 0;
     for (int e = e0; e < e1; ++e) {
+      const int blocks = (s_cnt[e] + ROW_TILE - 1) / ROW_TILE;
       sum += s_cnt[e];
-      psum += (s_cnt[e] + ROW_TILE - 1) / ROW_TILE * ROW_TILE;
+      psum += blocks * ROW_TILE;
+      tsum += (blocks + 1) >> 1;
     }
-    int isum = sum, ipsum = psum;
+    int isum = sum, ipsum = psum, itsum = tsum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int a = __shfl_up_sync(0xffffffffu, isum, o);
       const int b = __shfl_up_sync(0xffffffffu, ipsum, o);
+      const int c = __shfl_up_sync(0xffffffffu, itsum, o);
       if (lane >= o) {
         isum += a;
         ipsum += b;
+        itsum += c;
       }
     }
-    int off = isum - sum, poff = ipsum - psum;
+    int off = isum - sum, poff = ipsum - psum, toff = itsum - tsum;
     for (int e = e0; e < e1; ++e) {
+      const int blocks = (s_cnt[e] + ROW_TILE - 1) / ROW_TILE;
       s_off[e] = off;
       s_pad[e] = poff;
+      s_pair[e] = toff;
       off += s_cnt[e];
-      poff += (s_cnt[e] + ROW_TILE - 1) / ROW_TILE * ROW_TILE;
+      poff += blocks * ROW_TILE;
+      toff += (blocks + 1) >> 1;
     }
     if (lane == 31) {
       s_off[E_tgt] = isum;
       s_pad[E_tgt] = ipsum;
+      s_pair[E_tgt] = itsum;
     }
   }
   __syncthreads();
@@ -145,20 +154,21 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
       pp.pad_begin[e] = s_pad[e] + s_cnt[e];
     }
   }
-  const int n_tiles = s_pad[E_tgt] / ROW_TILE;
+  const int n_tiles = s_pair[E_tgt];
   if (tid == 0) {
-    *pp.n_m_tiles = n_tiles;
+    *pp.n_pair_tiles = n_tiles;
     *pp.ticket = 0u;  // ready for the next plan
   }
-  // expert of every 128-row tile: the last e with pad_offsets[e] <= first row of the tile
+  // expert and first row of every 256-row tile: the last e with s_pair[e] <= t owns tile t
   for (int t = tid; t < n_tiles; t += PLAN_THREADS) {
-    const int row = t * ROW_TILE;
-    int lo = 0, hi = E_tgt;  // invariant: s_pad[lo] <= row < s_pad[hi]
+    int lo = 0, hi = E_tgt;  // invariant: s_pair[lo] <= t < s_pair[hi]
     while (hi - lo > 1) {
       const int mid = (lo + hi) >> 1;
-      if (s_pad[mid] <= row) lo = mid; else hi = mid;
+      if (s_pair[mid] <= t) lo = mid; else hi = mid;
     }
-    pp.tile_expert[t] = lo;
+    const int row0 = s_pad[lo] + (t - s_pair[lo]) * 2 * ROW_TILE;
+    pp.pair_row0[t] = row0;
+    pp.pair_expert[t] = lo | (row0 + ROW_TILE < s_pad[lo + 1] ? PAIR_VALID2 : 0);
   }
   // pad rows carry no slot
   for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
@@ -222,7 +232,7 @@ static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, c
   const int R = (int)ctx->R, E = dm.E_tgt;
   const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
   if (phase == 0) {
-    const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 3 * E + 3) ? PLAN_WARPS * E : 3 * E + 3);
+    const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 4 * E + 4) ? PLAN_WARPS * E : 4 * E + 4);
     plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
   } else {
     const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
@@ -270,12 +280,13 @@ constexpr int NA_PAD_BEGIN = NA_ROW_SHIFT + 256;                      // [E]
 constexpr int NA_N_TILES = NA_PAD_BEGIN + 256;                        // [1]
 constexpr int NA_TICKET = NA_N_TILES + 64;                            // [1]
 constexpr int NA_STATUS = NA_TICKET + 64;                             // [1] used when the caller passes no status word
-constexpr int NA_TILE_EXPERT = NA_STATUS + 64;                        // [rows/128]
-constexpr int NA_SLOT_TO_PROW = NA_TILE_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE;   // [R]
+constexpr int NA_PAIR_ROW0 = NA_STATUS + 64;                          // [rows/128]
+constexpr int NA_PAIR_EXPERT = NA_PAIR_ROW0 + NOALLOC_MAX_ROWS / ROW_TILE;     // [rows/128]
+constexpr int NA_SLOT_TO_PROW = NA_PAIR_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE;  // [R]
 constexpr int NA_PROW_TO_SLOT = NA_SLOT_TO_PROW + NOALLOC_MAX_R;      // [rows]
 constexpr int NA_BLK_PREFIX = NA_PROW_TO_SLOT + NOALLOC_MAX_ROWS;     // [E * blocks]
 constexpr int NA_WORDS = NA_BLK_PREFIX + NOALLOC_MAX_E * NOALLOC_MAX_BLOCKS;
-static_assert(NA_TILE_EXPERT % 64 == 0 && NA_SLOT_TO_PROW % 64 == 0 && NA_PROW_TO_SLOT % 64 == 0 && NA_BLK_PREFIX % 64 == 0,
+static_assert(NA_PAIR_ROW0 % 64 == 0 && NA_PAIR_EXPERT % 64 == 0 && NA_SLOT_TO_PROW % 64 == 0 && NA_PROW_TO_SLOT % 64 == 0 && NA_BLK_PREFIX % 64 == 0,
               "scratch parts must start on 256-byte boundaries");
 
 // About 4.6 MB per GPU.  In host code this name is only a handle for cudaGetSymbolAddress: it is not a
@@ -336,10 +347,11 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.pp.pad_offsets = base + NA_PAD_OFFSETS;
   c.pp.row_shift = base + NA_ROW_SHIFT;
   c.pp.pad_begin = base + NA_PAD_BEGIN;
-  c.pp.n_m_tiles = base + NA_N_TILES;
+  c.pp.n_pair_tiles = base + NA_N_TILES;
   c.pp.ticket = reinterpret_cast<unsigned int*>(base + NA_TICKET);
   c.pp.status = status ? status : base + NA_STATUS;
-  c.pp.tile_expert = base + NA_TILE_EXPERT;
+  c.pp.pair_row0 = base + NA_PAIR_ROW0;
+  c.pp.pair_expert = base + NA_PAIR_EXPERT;
   c.pp.slot_to_prow = base + NA_SLOT_TO_PROW;
   c.pp.prow_to_slot = base + NA_PROW_TO_SLOT;
   c.pp.blk_prefix = base + NA_BLK_PREFIX;
