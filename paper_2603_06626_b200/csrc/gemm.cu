@@ -12,7 +12,7 @@
 // Tile: 256 x 256 x 64 per CTA pair (a cluster of two CTAs on neighbouring SMs, one pair-wide tcgen05.mma with
 // M = 256).  Each CTA owns 128 rows of the tile and half of B's 256 columns, so per 64-deep k-step it stages
 // 16 KB of A and 16 KB of B: a third less operand traffic per FLOP than a one-CTA 128 x 256 tile and room for a
-// 6-stage ring.  In every CTA warp 0 issues its TMA tile loads (128-byte swizzle; the byte counts of both CTAs
+// 5-stage ring.  In every CTA warp 0 issues its TMA tile loads (128-byte swizzle; the byte counts of both CTAs
 // complete on the leader CTA's barrier); warp 1 of the leader CTA issues the MMAs for the pair into one of two
 // 256-column TMEM accumulators (present in both CTAs) and releases stages / publishes accumulators to both
 // CTAs with multicast commits; warps 2-9 of each CTA drain the other accumulator with tcgen05.ld and run the
@@ -31,15 +31,15 @@ constexpr int BM = 128;                         // rows of the tile owned by one
 constexpr int PM = 2 * BM;                      // rows of the pair's tile
 constexpr int BN = 256, BK = 64;
 constexpr int BNH = BN / 2;                     // B columns staged by one CTA
-constexpr int STAGES = 6;
+constexpr int STAGES = 5;
 constexpr int A_BYTES = BM * BK * 2;            // 16 KB
 constexpr int B_BYTES = BNH * BK * 2;           // 16 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 32 KB per CTA and stage
 constexpr int ATOM_BYTES = 64 * BK * 2;         // one 64x64 bf16 box = 8 KB
 constexpr int EPI_WARPS = 8;                    // two warps per TMEM lane quadrant, each takes half of the columns
 constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;
-constexpr int EPI_STAGE_BYTES = 32 * 128;       // per epilogue warp: 32 rows x 128 bytes
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int EPI_STAGE_BYTES = 32 * 128;       // one staging block: 32 rows x 128 bytes; two per epilogue warp
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + EPI_WARPS * 2 * EPI_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct GemmParams {
@@ -176,8 +176,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // The dynamic shared memory starts at the same offset in both CTAs of the pair, so every address derived
   // below names the same location in either CTA (the MMA descriptors and multicast commits rely on that).
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t stage_base = smem_base + STAGES * STAGE_BYTES;          // epilogue staging, 4 KB per warp
-  const uint32_t bar_base = stage_base + EPI_WARPS * EPI_STAGE_BYTES;
+  const uint32_t stage_base = smem_base + STAGES * STAGE_BYTES;          // epilogue staging, 2 x 4 KB per warp
+  const uint32_t bar_base = stage_base + EPI_WARPS * 2 * EPI_STAGE_BYTES;
   // barriers (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
   //   full[s]       leader only: one arrival (leader's producer, with the byte count of BOTH CTAs' loads)
   //   empty[s]      each CTA: one arrival per round, delivered to both CTAs by the leader's multicast commit
@@ -323,143 +323,166 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     __syncwarp();
   } else {
-    // ===================== epilogue (warps 2..9) =====================
-    // Thread (quad, lane) owns tile row quad*32 + lane; the warp drains the 128 accumulator columns of
-    // its half.  Results go through a warp-private 32-row x 128-byte staging block in shared memory
-    // (128-byte swizzle, conflict-free) and leave as TMA tile stores: full 128-byte lines, clipped at
-    // the tensor bounds, so no store is masked by hand.
+    // ===================== epilogue (warps 2..9 of both CTAs) =====================
+    // Thread (quad, lane) owns row quad*32 + lane of this CTA's 128 rows; the warp drains the 128 accumulator
+    // columns of its half.  Results go through two warp-private 32-row x 128-byte staging blocks in shared
+    // memory (128-byte swizzle, conflict-free) and leave as TMA tile stores: full 128-byte lines, clipped at the
+    // tensor bounds, so no store is masked by hand.  Each store is its own bulk group and the blocks alternate,
+    // so a block is free again once all but the newest group have been read out of shared memory.
     const int quad = warp & 3;            // TMEM lane quadrant this warp may read
     const int half = (warp - 2) >> 2;     // which half of the tile's columns this warp drains
-    const int r = quad * 32 + lane;       // row of the tile owned by this thread
-    const uint32_t stage_buf = stage_base + (uint32_t)(warp - 2) * EPI_STAGE_BYTES;
-    const uint32_t my_row = stage_buf + (uint32_t)lane * 128u;
+    const int r = quad * 32 + lane;       // row of this CTA's block owned by this thread
+    const uint32_t blk_a = stage_base + (uint32_t)(warp - 2) * (2 * EPI_STAGE_BYTES);
+    const uint32_t blk_b = blk_a + EPI_STAGE_BYTES;
+    const uint32_t row_off = (uint32_t)lane * 128u;
     const uint32_t sw = (uint32_t)(lane & 7);
-    auto stage_open = [&]() {             // the previous store out of this block has been read
+    auto stage_wait_all = [&]() {         // every store issued so far has been read out of shared memory
       if (lane == 0) ptx::bulk_wait_read0();
       __syncwarp();
     };
-    auto stage_put = [&](int q, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {  // 16-byte unit q of this row
-      ptx::st_shared_v4(my_row + (((uint32_t)q ^ sw) << 4), a, b, c, d);
+    auto stage_wait_older = [&]() {       // ... every store but the newest
+      if (lane == 0) ptx::bulk_wait_read1();
+      __syncwarp();
     };
-    auto stage_put_bf16 = [&](int q0, const float (&v)[32]) {  // 32 fp32 -> 4 units of 8 bf16
+    auto stage_put = [&](uint32_t blk, int q, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {  // 16-byte unit q of this row
+      ptx::st_shared_v4(blk + row_off + (((uint32_t)q ^ sw) << 4), a, b, c, d);
+    };
+    auto stage_put_bf16 = [&](uint32_t blk, int q0, const float (&v)[32]) {  // 32 fp32 -> 4 units of 8 bf16
 #pragma unroll
       for (int q = 0; q < 4; ++q)
-        stage_put(q0 + q, pack_bf16(v[q * 8 + 0], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
+        stage_put(blk, q0 + q, pack_bf16(v[q * 8 + 0], v[q * 8 + 1]), pack_bf16(v[q * 8 + 2], v[q * 8 + 3]),
                   pack_bf16(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16(v[q * 8 + 6], v[q * 8 + 7]));
     };
-    auto stage_send_2d = [&](const CUtensorMap* tm, int x, int y) {
+    auto stage_send_2d = [&](uint32_t blk, const CUtensorMap* tm, int x, int y) {
       ptx::fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        ptx::tma_store_2d(tm, stage_buf, x, y);
+        ptx::tma_store_2d(tm, blk, x, y);
         ptx::bulk_commit();
       }
     };
-    auto stage_send_3d = [&](const CUtensorMap* tm, int x, int y, int z) {
+    auto stage_send_3d = [&](uint32_t blk, const CUtensorMap* tm, int x, int y, int z) {
       ptx::fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        ptx::tma_store_3d(tm, stage_buf, x, y, z);
+        ptx::tma_store_3d(tm, blk, x, y, z);
         ptx::bulk_commit();
       }
     };
+    // DH: saved pre-activations G and U of one 32-column chunk of this thread's row (zeros beyond F)
+    auto load_gu = [&](const Tile& ti, int c, uint4 (&g4)[4], uint4 (&u4)[4]) {
+      const int c0 = half * 128 + c * 32;
+      const int n_left = ti.m_valid > 0 ? ti.n_valid - c0 : 0;
+      const size_t gi = ((size_t)ti.row0 + r) * p.F + ti.col0 + c0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (q * 8 < n_left) {
+          g4[q] = *reinterpret_cast<const uint4*>(p.in_G + gi + q * 8);
+          u4[q] = *reinterpret_cast<const uint4*>(p.in_U + gi + q * 8);
+        } else {
+          g4[q] = make_uint4(0u, 0u, 0u, 0u);
+          u4[q] = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    };
+    const uint32_t leader_tempty[2] = {ptx::map_to_cta(tempty_bar(0), 0), ptx::map_to_cta(tempty_bar(1), 0)};
     int acc = 0;
     uint32_t acc_ph = 0;
-    const uint32_t leader_tempty[2] = {ptx::map_to_cta(tempty_bar(0), 0), ptx::map_to_cta(tempty_bar(1), 0)};
+    uint32_t flip = 0;                    // staging block the next single-block store uses (they strictly alternate)
     for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
       const Tile ti = decode_tile<MODE>(p, t, rank);
+      const bool live = ti.m_valid > 0;    // false: this CTA only lent its half of B to the pair
+      uint4 g4[4], u4[4];
+      if (MODE == MODE_DH) load_gu(ti, 0, g4, u4);   // in flight while the main loop of this tile finishes
       if (!ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag)) break;
       ptx::tc_fence_after();
       const uint32_t t_row = tmem_base + (uint32_t)acc * BN + ((uint32_t)(quad * 32) << 16);
       const bool have_acc = ti.num_k > 0;
       const int y0 = ti.row0 + quad * 32;  // first output row of this warp's block
 
-      const bool live = ti.m_valid > 0;    // false: this CTA only lent its half of B to the pair
       if (MODE == MODE_UP) {
         // accumulator columns 0..127 = gate, 128..255 = up, for F-columns col0..col0+127; this warp: 64 of them
         if (live && ti.n_valid - half * 64 > 0) {
           const float g = gate_of_row(p, ti.row0 + r);
-          uint32_t pg[32], pu[32], ph[32];   // packed bf16 pairs: 64 columns each
+          const int x = ti.col0 + half * 64;
+          uint32_t ph[32];                 // H' of the 64 columns, packed bf16 pairs
 #pragma unroll
           for (int cc = 0; cc < 2; ++cc) {
             uint32_t rg[32], ru[32];
             ptx::tmem_ld32(t_row + half * 64 + cc * 32, rg);
             ptx::tmem_ld32(t_row + 128 + half * 64 + cc * 32, ru);
             ptx::tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float g0 = __uint_as_float(rg[i]), g1 = __uint_as_float(rg[i + 1]);
-              const float u0 = __uint_as_float(ru[i]), u1 = __uint_as_float(ru[i + 1]);
-              const float s0 = __fdividef(1.f, 1.f + __expf(-g0)), s1 = __fdividef(1.f, 1.f + __expf(-g1));
-              pg[cc * 16 + i / 2] = pack_bf16(g0, g1);
-              pu[cc * 16 + i / 2] = pack_bf16(u0, u1);
-              ph[cc * 16 + i / 2] = pack_bf16(g * g0 * s0 * u0, g * g1 * s1 * u1);
-            }
-          }
-          const int x = ti.col0 + half * 64;
-          stage_open();
-#pragma unroll
-          for (int q = 0; q < 8; ++q) stage_put(q, pg[q * 4], pg[q * 4 + 1], pg[q * 4 + 2], pg[q * 4 + 3]);
-          stage_send_2d(&tmC0, x, y0);
-          stage_open();
-#pragma unroll
-          for (int q = 0; q < 8; ++q) stage_put(q, pu[q * 4], pu[q * 4 + 1], pu[q * 4 + 2], pu[q * 4 + 3]);
-          stage_send_2d(&tmC1, x, y0);
-          stage_open();
-#pragma unroll
-          for (int q = 0; q < 8; ++q) stage_put(q, ph[q * 4], ph[q * 4 + 1], ph[q * 4 + 2], ph[q * 4 + 3]);
-          stage_send_2d(&tmC2, x, y0);
-        }
-      } else if (MODE == MODE_DOWN || MODE == MODE_DX) {
-        for (int blk = 0; blk < 2; ++blk) {          // two 64-column blocks per warp
-          const int cb = half * 128 + blk * 64;
-          if (!live || ti.n_valid - cb <= 0) break;
-          stage_open();
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            uint32_t ra[32];
-            ptx::tmem_ld32(t_row + cb + cc * 32, ra);
-            ptx::tmem_ld_wait();
-            float v[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
-            stage_put_bf16(cc * 4, v);
-          }
-          stage_send_2d(&tmC0, ti.col0 + cb, y0);
-        }
-      } else if (MODE == MODE_DH) {
-        const size_t prow = (size_t)ti.row0 + r;
-        const float g = live ? gate_of_row(p, (int)prow) : 0.f;
-        const size_t gi = prow * p.F + ti.col0;
-        float dgate = 0.f;
-        for (int blk = 0; blk < 2; ++blk) {
-          const int cb = half * 128 + blk * 64;
-          if (!live || ti.n_valid - cb <= 0) break;
-          uint32_t pdg[32], pdu[32];
-#pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
-            const int c0 = cb + cc * 32;
-            const int n_left = ti.n_valid - c0;
-            // saved pre-activations of this chunk: issue the loads before waiting on TMEM
-            uint4 g4[4], u4[4];
+            if (cc == 0) stage_wait_all();
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              if (q * 8 < n_left) {
-                g4[q] = *reinterpret_cast<const uint4*>(p.in_G + gi + c0 + q * 8);
-                u4[q] = *reinterpret_cast<const uint4*>(p.in_U + gi + c0 + q * 8);
-              } else {
-                g4[q] = make_uint4(0u, 0u, 0u, 0u);
-                u4[q] = make_uint4(0u, 0u, 0u, 0u);
+              uint32_t wg[4], wu[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int c = q * 8 + 2 * i;
+                const float g0 = __uint_as_float(rg[c]), g1 = __uint_as_float(rg[c + 1]);
+                const float u0 = __uint_as_float(ru[c]), u1 = __uint_as_float(ru[c + 1]);
+                const float s0 = __fdividef(1.f, 1.f + __expf(-g0)), s1 = __fdividef(1.f, 1.f + __expf(-g1));
+                wg[i] = pack_bf16(g0, g1);
+                wu[i] = pack_bf16(u0, u1);
+                ph[cc * 16 + q * 4 + i] = pack_bf16(g * g0 * s0 * u0, g * g1 * s1 * u1);
               }
+              stage_put(blk_a, cc * 4 + q, wg[0], wg[1], wg[2], wg[3]);
+              stage_put(blk_b, cc * 4 + q, wu[0], wu[1], wu[2], wu[3]);
             }
+          }
+          stage_send_2d(blk_a, &tmC0, x, y0);
+          stage_send_2d(blk_b, &tmC1, x, y0);
+          stage_wait_older();              // block a has been read (the store of block b may still be reading)
+#pragma unroll
+          for (int q = 0; q < 8; ++q) stage_put(blk_a, q, ph[q * 4], ph[q * 4 + 1], ph[q * 4 + 2], ph[q * 4 + 3]);
+          stage_send_2d(blk_a, &tmC2, x, y0);
+        }
+      } else if (MODE == MODE_DOWN || MODE == MODE_DX) {
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk) {          // two 64-column blocks per warp, one staging block each
+          const int cb = half * 128 + blk * 64;
+          if (live && ti.n_valid - cb > 0) {
+            const uint32_t sb = flip ? blk_b : blk_a;   // not the block of the previous store
+            flip ^= 1u;
+#pragma unroll
+            for (int cc = 0; cc < 2; ++cc) {
+              uint32_t ra[32];
+              ptx::tmem_ld32(t_row + cb + cc * 32, ra);
+              ptx::tmem_ld_wait();
+              if (cc == 0) stage_wait_older();
+              float v[32];
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
+              stage_put_bf16(sb, cc * 4, v);
+            }
+            stage_send_2d(sb, &tmC0, ti.col0 + cb, y0);
+          }
+        }
+      } else if (MODE == MODE_DH) {
+        const float g = live ? gate_of_row(p, ti.row0 + r) : 0.f;
+        float dgate = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {                // four 32-column chunks; chunks 2c, 2c+1 fill one pair of blocks
+          const int cb = half * 128 + (c >> 1) * 64; // first column of the 64-column block
+          const int c0 = half * 128 + c * 32;
+          const int n_left = live ? ti.n_valid - c0 : 0;
+          uint4 cg[4], cu[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            cg[q] = g4[q];
+            cu[q] = u4[q];
+          }
+          if (c < 3) load_gu(ti, c + 1, g4, u4);     // next chunk's loads fly during this chunk's arithmetic
+          if (n_left > 0) {
             uint32_t ra[32];
             ptx::tmem_ld32(t_row + c0, ra);
             ptx::tmem_ld_wait();
+            if ((c & 1) == 0) stage_wait_all();
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               float fg[8], fu[8], vdg[8], vdu[8];
-              unpack8(g4[q], fg);
-              unpack8(u4[q], fu);
+              unpack8(cg[q], fg);
+              unpack8(cu[q], fu);
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const float dA = (q * 8 < n_left) ? __uint_as_float(ra[q * 8 + i]) : 0.f;
@@ -470,41 +493,43 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 vdg[i] = dH * fu[i] * sg * (1.f + fg[i] * (1.f - sg));
                 vdu[i] = dH * si;
               }
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                pdg[cc * 16 + q * 4 + i] = pack_bf16(vdg[2 * i], vdg[2 * i + 1]);
-                pdu[cc * 16 + q * 4 + i] = pack_bf16(vdu[2 * i], vdu[2 * i + 1]);
-              }
+              stage_put(blk_a, (c & 1) * 4 + q, pack_bf16(vdg[0], vdg[1]), pack_bf16(vdg[2], vdg[3]), pack_bf16(vdg[4], vdg[5]),
+                        pack_bf16(vdg[6], vdg[7]));
+              stage_put(blk_b, (c & 1) * 4 + q, pack_bf16(vdu[0], vdu[1]), pack_bf16(vdu[2], vdu[3]), pack_bf16(vdu[4], vdu[5]),
+                        pack_bf16(vdu[6], vdu[7]));
             }
           }
-          stage_open();
-#pragma unroll
-          for (int q = 0; q < 8; ++q) stage_put(q, pdg[q * 4], pdg[q * 4 + 1], pdg[q * 4 + 2], pdg[q * 4 + 3]);
-          stage_send_2d(&tmC0, ti.col0 + cb, y0);   // dG: columns [0,F) of [dG|dU]
-          stage_open();
-#pragma unroll
-          for (int q = 0; q < 8; ++q) stage_put(q, pdu[q * 4], pdu[q * 4 + 1], pdu[q * 4 + 2], pdu[q * 4 + 3]);
-          stage_send_2d(&tmC1, ti.col0 + cb, y0);   // dU: columns [F,2F)
+          // after the second chunk of a block pair (or the last valid one): ship dG and dU of these 64 columns
+          if ((c & 1) == 1 && live && ti.n_valid - cb > 0) {
+            stage_send_2d(blk_a, &tmC0, ti.col0 + cb, y0);   // dG: columns [0,F) of [dG|dU]
+            stage_send_2d(blk_b, &tmC1, ti.col0 + cb, y0);   // dU: columns [F,2F)
+          }
         }
-        const int nt = ti.col0 / BN;
-        if (live) p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + prow] = dgate;
+        if (live) {
+          const int nt = ti.col0 / BN;
+          p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + (size_t)ti.row0 + r] = dgate;
+        }
       } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile, four 32-column blocks per warp
         if (y0 < ti.row0 + ti.m_valid) {
+#pragma unroll
           for (int blk = 0; blk < 4; ++blk) {
             const int cb = half * 128 + blk * 32;
-            if (ti.n_valid - cb <= 0) break;
-            uint32_t ra[32];
-            if (have_acc) {
-              ptx::tmem_ld32(t_row + cb, ra);
-              ptx::tmem_ld_wait();
-            } else {
+            if (ti.n_valid - cb > 0) {
+              const uint32_t sb = flip ? blk_b : blk_a;   // not the block of the previous store
+              flip ^= 1u;
+              uint32_t ra[32];
+              if (have_acc) {
+                ptx::tmem_ld32(t_row + cb, ra);
+                ptx::tmem_ld_wait();
+              } else {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) ra[i] = 0u;
+                for (int i = 0; i < 32; ++i) ra[i] = 0u;
+              }
+              stage_wait_older();
+#pragma unroll
+              for (int q = 0; q < 8; ++q) stage_put(sb, q, ra[q * 4], ra[q * 4 + 1], ra[q * 4 + 2], ra[q * 4 + 3]);
+              stage_send_3d(sb, &tmC0, ti.col0 + cb, y0, ti.e);
             }
-            stage_open();
-#pragma unroll
-            for (int q = 0; q < 8; ++q) stage_put(q, ra[q * 4], ra[q * 4 + 1], ra[q * 4 + 2], ra[q * 4 + 3]);
-            stage_send_3d(&tmC0, ti.col0 + cb, y0, ti.e);
           }
         }
       }

@@ -14,6 +14,8 @@ namespace grouter {
 
 constexpr int MOVE_THREADS = 256;
 constexpr int MOVE_WARPS = MOVE_THREADS / 32;
+constexpr int SCATTER_SEG = 8;
+constexpr int REDUCE_SEG = 8;
 
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
   uint4 v;
@@ -24,6 +26,8 @@ __device__ __forceinline__ void st_v4(void* p, const uint4& v) {
   asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+// SEG: 16-byte units each lane holds per pass; a warp moves SEG * 512 contiguous bytes of a row at a time.
+template <int SEG>
 __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
                                                                     const int32_t* __restrict__ slot_to_prow,
                                                                     const int32_t* __restrict__ pad_begin,
@@ -35,10 +39,10 @@ __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_b
   for (int t = gwarp; t < T; t += nwarps) {
     const int my_prow = lane < k ? __ldg(slot_to_prow + (size_t)t * k + lane) : 0;
     const char* s = reinterpret_cast<const char*>(src + (size_t)t * d);
-    for (int u0 = 0; u0 < units; u0 += 128) {
-      uint4 v[4];
+    for (int u0 = 0; u0 < units; u0 += 32 * SEG) {
+      uint4 v[SEG];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
+      for (int i = 0; i < SEG; ++i) {
         const int u = u0 + i * 32 + lane;
         if (u < units) v[i] = ld_nc_v4(s + (size_t)u * 16);
       }
@@ -46,7 +50,7 @@ __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_b
         const int prow = __shfl_sync(0xffffffffu, my_prow, j);
         char* o = reinterpret_cast<char*>(dst + (size_t)prow * d);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < SEG; ++i) {
           const int u = u0 + i * 32 + lane;
           if (u < units) st_v4(o + (size_t)u * 16, v[i]);
         }
@@ -74,6 +78,9 @@ __device__ __forceinline__ void acc_bf16x8(float (&a)[8], const uint4& v) {
   }
 }
 
+// SEG: 16-byte units each lane accumulates per pass.  A warp reads SEG * 512 contiguous bytes of one routed row
+// before it moves to the next row, so DRAM sees long sequential bursts instead of many interleaved short ones.
+template <int SEG>
 __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ out,
                                                                    const int32_t* __restrict__ slot_to_prow, int T, int k, int d,
                                                                    const float* __restrict__ dgate_part, int n_part, size_t part_stride,
@@ -90,30 +97,37 @@ __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bf
       dgates[(size_t)t * k + lane] = g;
     }
     char* o = reinterpret_cast<char*>(out + (size_t)t * d);
-    for (int u0 = 0; u0 < units; u0 += 64) {
-      float a0[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      float a1[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      const int ua = u0 + lane, ub = u0 + 32 + lane;
-#pragma unroll 4
-      for (int j = 0; j < k; ++j) {
+    for (int u0 = 0; u0 < units; u0 += 32 * SEG) {
+      float acc[SEG][8];
+#pragma unroll
+      for (int i = 0; i < SEG; ++i)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[i][c] = 0.f;
+      for (int j = 0; j < k; ++j) {          // slot order: the sum is deterministic
         const int prow = __shfl_sync(0xffffffffu, my_prow, j);
         const char* s = reinterpret_cast<const char*>(src + (size_t)prow * d);
-        if (ua < units) acc_bf16x8(a0, ld_nc_v4(s + (size_t)ua * 16));
-        if (ub < units) acc_bf16x8(a1, ld_nc_v4(s + (size_t)ub * 16));
-      }
-      if (ua < units) {
-        uint4 v;
-        __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+        uint4 v[SEG];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(a0[2 * i], a0[2 * i + 1]);
-        st_v4(o + (size_t)ua * 16, v);
-      }
-      if (ub < units) {
-        uint4 v;
-        __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+        for (int i = 0; i < SEG; ++i) {
+          const int u = u0 + i * 32 + lane;
+          if (u < units) v[i] = ld_nc_v4(s + (size_t)u * 16);
+        }
 #pragma unroll
-        for (int i = 0; i < 4; ++i) p[i] = __floats2bfloat162_rn(a1[2 * i], a1[2 * i + 1]);
-        st_v4(o + (size_t)ub * 16, v);
+        for (int i = 0; i < SEG; ++i) {
+          const int u = u0 + i * 32 + lane;
+          if (u < units) acc_bf16x8(acc[i], v[i]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < SEG; ++i) {
+        const int u = u0 + i * 32 + lane;
+        if (u < units) {
+          uint4 v;
+          __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) p[c] = __floats2bfloat162_rn(acc[i][2 * c], acc[i][2 * c + 1]);
+          st_v4(o + (size_t)u * 16, v);
+        }
       }
     }
   }
@@ -127,7 +141,7 @@ static int mover_grid(const grouter_ctx* ctx, int T) {
 
 cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  scatter_rows_kernel<<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_prow, ctx->pp.pad_begin,
+  scatter_rows_kernel<SCATTER_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_prow, ctx->pp.pad_begin,
                                                                       ctx->pp.pad_offsets, dm.T, dm.k, dm.d, dm.E_tgt);
   return cudaGetLastError();
 }
@@ -135,7 +149,7 @@ cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv
 cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part, int n_part,
                                float* dgates, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  reduce_rows_kernel<<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_prow, dm.T, dm.k, dm.d, dgate_part, n_part,
+  reduce_rows_kernel<REDUCE_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_prow, dm.T, dm.k, dm.d, dgate_part, n_part,
                                                                      (size_t)ctx->R_pad_max, dgates);
   return cudaGetLastError();
 }
