@@ -50,10 +50,13 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def kernel_work(w: synth.Workload):
+def kernel_work(w: synth.Workload, counts: np.ndarray):
     """Algorithmic work per launch: FLOPs over valid routed rows only (padding earns nothing) for the
-    GEMMs; bytes (T + R) * d * 2 for the row movers; plan: ids read, two permutations written."""
+    GEMMs; bytes (T + R) * d * 2 for the row movers; plan: ids read, two permutations written; the zero-fill
+    writes the fp32 gradients of the experts whose rows are contracted in several chunks (more than 4096
+    padded rows)."""
     R, d, F, T = w.R, w.d, w.ffn, w.T
+    n_split = int((((counts + 127) // 128) * 128 > 4096).sum())
     dF = 2.0 * R * d * F
     idb = 1 if w.E_src <= 256 else 4
     return {
@@ -62,6 +65,7 @@ def kernel_work(w: synth.Workload):
         "gather_X": ("byte", (T + R) * d * 2.0), "combine_Y": ("byte", (T + R) * d * 2.0),
         "gather_dY": ("byte", (T + R) * d * 2.0), "reduce_dX": ("byte", (T + R) * d * 2.0),
         "plan_hist": ("byte", R * idb + 0.0), "plan_permute": ("byte", R * idb + 2.0 * R * 4),
+        "zero_split_dW": ("byte", n_split * 3.0 * d * F * 4),
     }
 
 
@@ -253,7 +257,7 @@ def main():
     layer.check_status()
     barrier()
     torch.cuda.synchronize()
-    layer.timing_enable(12 * args.steps)
+    layer.timing_enable(len(binding.KERNEL_SLOTS) * args.steps)
     wall0 = time.time()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
@@ -314,7 +318,7 @@ def main():
 
     # ---- roofline of the dominant kernel, and the per-kernel table ----
     peaks, peak_src = load_peaks()
-    work = kernel_work(w)
+    work = kernel_work(w, layer.counts.cpu().numpy().astype(np.int64))
     kernels = {}
     for name, (ms, n) in per_kernel.items():
         if n == 0:

@@ -145,7 +145,9 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
  *   dY     [T,d] bf16                 dX     [T,d] bf16 out
  *   dW_gu  [E_tgt, 2*ffn, d] f32 out  dW_d   [E_tgt, d, ffn] f32 out
  *   dgates [T,k] f32 out: dgates[t,j] = <dY[t,:], f_{e(t,j)}(X[t,:])> (gates are leaf inputs)
- * Experts that received no slot get exact zeros in dW_*.  Uses the workspace
+ * Experts that received no slot get exact zeros in dW_*.  An expert with more than 4096 rows is contracted in
+ * chunks of rows that are added into its gradient in no fixed order, so its dW_* may differ in the last bits
+ * from run to run; everything else (Y, dX, dgates, dW_* of smaller experts) is bit-reproducible.  Uses the workspace
  * contents left by the matching grouter_moe_fwd (else INVALID_STATE). */
 int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void* gates, const void* W_gu,
                     const void* W_d, void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace,
@@ -176,8 +178,8 @@ const char* grouter_strerror(int code);
  * elapsed milliseconds and launch counts per kernel slot, and empties the pool.
  * Slots: 0 plan_hist, 1 plan_permute, 2 gather_X, 3 gemm_up_swiglu, 4 gemm_down,
  * 5 combine_Y, 6 gather_dY, 7 gemm_dH, 8 wgrad_down, 9 gemm_dX, 10 wgrad_gate_up,
- * 11 reduce_dX.   total_ms, launches: HOST arrays of GROUTER_NUM_KERNELS entries. */
-#define GROUTER_NUM_KERNELS 12
+ * 11 reduce_dX, 12 zero_split_dW.   total_ms, launches: HOST arrays of GROUTER_NUM_KERNELS entries. */
+#define GROUTER_NUM_KERNELS 13
 int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records);
 int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t* launches);
 

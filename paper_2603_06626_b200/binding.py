@@ -21,7 +21,7 @@ EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grou
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
-                "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX"]
+                "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW"]
 
 
 class GrouterDims(ctypes.Structure):

@@ -154,6 +154,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->R = (int64_t)dims->T * dims->k;
   c->R_pad_max = r_pad_max(*dims);
   c->max_m_tiles = (int)(c->R_pad_max / ROW_TILE);
+  c->max_wchunks = dims->E_tgt + (int)(c->R_pad_max / WGRAD_KCHUNK) + 1;
   c->geom = plan_geom(c->R);
   c->planned = c->forwarded = false;
   c->ev_start = c->ev_stop = nullptr;
@@ -164,6 +165,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
   const size_t o_pad = take((size_t)(E + 1) * 4), o_shift = take((size_t)E * 4), o_pb = take((size_t)E * 4);
   const size_t o_pr = take((size_t)c->max_m_tiles * 4), o_pe = take((size_t)c->max_m_tiles * 4), o_nt = take(4), o_s2p = take((size_t)c->R * 4);
+  const size_t o_we = take((size_t)c->max_wchunks * 4), o_wr = take((size_t)c->max_wchunks * 4), o_wn = take((size_t)c->max_wchunks * 4), o_nw = take(4);
   const size_t o_p2s = take((size_t)c->R_pad_max * 4), o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
   if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
     delete c;
@@ -181,6 +183,10 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.pair_row0 = reinterpret_cast<int32_t*>(b + o_pr);
   c->pp.pair_expert = reinterpret_cast<int32_t*>(b + o_pe);
   c->pp.n_pair_tiles = reinterpret_cast<int32_t*>(b + o_nt);
+  c->pp.wchunk_expert = reinterpret_cast<int32_t*>(b + o_we);
+  c->pp.wchunk_row0 = reinterpret_cast<int32_t*>(b + o_wr);
+  c->pp.wchunk_rows = reinterpret_cast<int32_t*>(b + o_wn);
+  c->pp.n_wchunks = reinterpret_cast<int32_t*>(b + o_nw);
   c->pp.slot_to_prow = reinterpret_cast<int32_t*>(b + o_s2p);
   c->pp.prow_to_slot = reinterpret_cast<int32_t*>(b + o_p2s);
   c->pp.blk_prefix = reinterpret_cast<int32_t*>(b + o_bp);
@@ -260,6 +266,10 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
   {
     Timed tm(ctx, 7, st);
     if (launch_grouped_gemm(ctx, MODE_DH, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 12, st);
+    if (launch_zero_split_dw(ctx, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
   {
     Timed tm(ctx, 8, st);

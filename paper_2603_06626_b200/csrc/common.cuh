@@ -15,6 +15,10 @@ constexpr int STATUS_TIMEOUT = 2;
 
 constexpr int ROW_TILE = 128;        // rows one CTA owns in a GEMM tile; expert segments are padded to it
 constexpr int PAIR_VALID2 = 1 << 30; // flag in PaddedPlan::pair_expert
+// The weight-gradient GEMMs contract over an expert's rows in chunks of at most this many (padded) rows, so that
+// the operand rows of one chunk stay in L2 while every output tile of the expert reads them.
+constexpr int WGRAD_KCHUNK = 4096;
+constexpr int WCHUNK_SPLIT = 1 << 30; // flag in PaddedPlan::wchunk_expert: the expert has several chunks
 constexpr int PLAN_THREADS = 256;    // 8 warps per plan block
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
 constexpr int PLAN_MIN_CHUNK = 2048; // slots per plan block (lower bound)
@@ -46,6 +50,12 @@ struct PaddedPlan {
   int32_t* pair_row0;     // [max_m_tiles] first padded row of each 256-row tile
   int32_t* pair_expert;   // [max_m_tiles] expert of the tile; bit 30 set when the second half holds rows of that expert
   int32_t* n_pair_tiles;  // [1]
+  // Work list of the weight-gradient GEMMs: one entry per (expert, chunk of rows).  An expert with several
+  // chunks accumulates them into its pre-zeroed gradient with reduce-add stores; a one-chunk expert stores.
+  int32_t* wchunk_expert; // [max_wchunks] expert | WCHUNK_SPLIT
+  int32_t* wchunk_row0;   // [max_wchunks] first padded row of the chunk
+  int32_t* wchunk_rows;   // [max_wchunks] rows in the chunk (multiple of 128; 0 for an expert without slots)
+  int32_t* n_wchunks;     // [1]
   int32_t* slot_to_prow;  // [R]
   int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows
   int32_t* blk_prefix;    // [E_tgt * nblk] per-block histogram, then exclusive prefix over blocks
@@ -61,6 +71,7 @@ struct grouter_ctx {
   int64_t R;
   int64_t R_pad_max;      // round_up(R,128) + 128*E_tgt
   int max_m_tiles;
+  int max_wchunks;        // E_tgt + R_pad_max / WGRAD_KCHUNK + 1
   grouter::PlanGeom geom;
   grouter::PaddedPlan pp;
   void* d_block;          // one allocation backing pp
@@ -106,6 +117,8 @@ enum GemmMode { MODE_UP = 0, MODE_DOWN = 1, MODE_DH = 2, MODE_DX = 3, MODE_WGRAD
 
 cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace& ws, const void* gates, const void* W_gu,
                                 const void* W_d, float* dW_gu, float* dW_d, cudaStream_t st);
+// Zero-fills dW_gu[e] and dW_d[e] of every expert whose rows are split over several chunks.
+cudaError_t launch_zero_split_dw(grouter_ctx* ctx, float* dW_gu, float* dW_d, cudaStream_t st);
 cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,
                               cudaStream_t st);
 

@@ -47,7 +47,10 @@ struct GemmParams {
   const int32_t* n_pair_tiles; // device scalar: 256-row tiles in use (row-parallel modes)
   const int32_t* pair_row0;    // device [tiles] first padded row
   const int32_t* pair_expert;  // device [tiles] expert | PAIR_VALID2
-  const int32_t* pad_offsets;  // device [E+1]
+  const int32_t* n_wchunks;    // device scalar: (expert, row chunk) entries (weight-gradient modes)
+  const int32_t* wchunk_expert;// device [chunks] expert | WCHUNK_SPLIT
+  const int32_t* wchunk_row0;  // device [chunks] first padded row
+  const int32_t* wchunk_rows;  // device [chunks] rows, multiple of 128
   int32_t E, d, F;
   int32_t M, N, K;             // DENSE: problem; WGRAD: per-expert output M x N
   int32_t tiles_m, tiles_n;    // output tiles per problem (tiles_m unused by row-parallel modes)
@@ -69,11 +72,12 @@ struct Tile {     // one CTA's share of a pair tile
   int row0, col0; // origin of this CTA's 128 x 256 output block within the output matrix of this problem
   int e;
   int m_valid, n_valid;   // m_valid <= 0: this CTA's rows are not part of the problem (it still feeds its B half)
+  bool add;               // weight gradients: the tile is one of several partial sums added into a zeroed output
 };
 
 template <int MODE>
 __device__ __forceinline__ int total_tiles(const GemmParams& p) {
-  if (MODE == MODE_WGRAD_D || MODE == MODE_WGRAD_GU) return p.E * p.tiles_m * p.tiles_n;
+  if (MODE == MODE_WGRAD_D || MODE == MODE_WGRAD_GU) return __ldg(p.n_wchunks) * p.tiles_m * p.tiles_n;
   if (MODE == MODE_DENSE) return p.tiles_m * p.tiles_n;
   return __ldg(p.n_pair_tiles) * p.tiles_n;
 }
@@ -82,6 +86,7 @@ __device__ __forceinline__ int total_tiles(const GemmParams& p) {
 template <int MODE>
 __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank) {
   Tile ti;
+  ti.add = false;
   if (MODE == MODE_UP || MODE == MODE_DOWN || MODE == MODE_DH || MODE == MODE_DX) {
     const int mt = t / p.tiles_n, nt = t - mt * p.tiles_n;
     const int pe = __ldg(p.pair_expert + mt);
@@ -89,7 +94,9 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
     ti.row0 = __ldg(p.pair_row0 + mt) + rank * BM;
     ti.m_valid = (rank == 0 || (pe & PAIR_VALID2)) ? BM : 0;
     ti.a_x = 0;
-    ti.a_y = ti.row0;
+    // a CTA without rows of its own loads its A block from beyond the last row: TMA fills zeros, which costs
+    // no memory traffic and keeps the unused half of the pair's MMA quiet
+    ti.a_y = ti.m_valid > 0 ? ti.row0 : (int)p.R_pad_max;
     if (MODE == MODE_UP) {          // B = W_gu as [E*2F, d], K-major; leader stages 128 gate rows, peer the 128 up rows
       ti.col0 = nt * 128;
       ti.n_valid = min(128, p.F - ti.col0);
@@ -116,11 +123,16 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
       ti.num_k = (2 * p.F + BK - 1) / BK;
     }
   } else if (MODE == MODE_WGRAD_D || MODE == MODE_WGRAD_GU) {
+    // all output tiles of one (expert, row chunk) are adjacent in the schedule: the CTA pairs in flight read the
+    // same chunk of operand rows, which therefore stays in L2 however long the expert's row list is
     const int per = p.tiles_m * p.tiles_n;
-    ti.e = t / per;
-    const int r = t - ti.e * per;
+    const int ci = t / per;
+    const int r = t - ci * per;
     const int mt = r / p.tiles_n, nt = r - mt * p.tiles_n;
-    const int k0 = __ldg(p.pad_offsets + ti.e), k1 = __ldg(p.pad_offsets + ti.e + 1);
+    const int we = __ldg(p.wchunk_expert + ci);
+    ti.e = we & ~WCHUNK_SPLIT;
+    ti.add = (we & WCHUNK_SPLIT) != 0;
+    const int k0 = __ldg(p.wchunk_row0 + ci), k1 = k0 + __ldg(p.wchunk_rows + ci);
     ti.row0 = mt * PM + rank * BM;
     ti.col0 = nt * BN;
     ti.m_valid = min(BM, p.M - ti.row0);
@@ -361,11 +373,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ptx::bulk_commit();
       }
     };
-    auto stage_send_3d = [&](uint32_t blk, const CUtensorMap* tm, int x, int y, int z) {
+    auto stage_send_3d = [&](uint32_t blk, const CUtensorMap* tm, int x, int y, int z, bool add) {
       ptx::fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        ptx::tma_store_3d(tm, blk, x, y, z);
+        if (add) ptx::tma_reduce_add_3d(tm, blk, x, y, z);
+        else ptx::tma_store_3d(tm, blk, x, y, z);
         ptx::bulk_commit();
       }
     };
@@ -528,7 +541,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               stage_wait_older();
 #pragma unroll
               for (int q = 0; q < 8; ++q) stage_put(sb, q, ra[q * 4], ra[q * 4 + 1], ra[q * 4 + 2], ra[q * 4 + 3]);
-              stage_send_3d(sb, &tmC0, ti.col0 + cb, y0, ti.e);
+              stage_send_3d(sb, &tmC0, ti.col0 + cb, y0, ti.e, ti.add);
             }
           }
         }
@@ -638,7 +651,10 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.n_pair_tiles = ctx->pp.n_pair_tiles;
   p.pair_row0 = ctx->pp.pair_row0;
   p.pair_expert = ctx->pp.pair_expert;
-  p.pad_offsets = ctx->pp.pad_offsets;
+  p.n_wchunks = ctx->pp.n_wchunks;
+  p.wchunk_expert = ctx->pp.wchunk_expert;
+  p.wchunk_row0 = ctx->pp.wchunk_row0;
+  p.wchunk_rows = ctx->pp.wchunk_rows;
   p.E = E;
   p.d = d;
   p.F = F;
@@ -697,6 +713,33 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
     default:
       return cudaErrorInvalidValue;
   }
+}
+
+// Zero-fill of the gradients that the weight-gradient GEMMs build up from several partial sums.
+__global__ void __launch_bounds__(256) zero_split_dw_kernel(const int32_t* __restrict__ n_wchunks, const int32_t* __restrict__ wchunk_expert,
+                                                            const int32_t* __restrict__ wchunk_row0, const int32_t* __restrict__ pad_offsets,
+                                                            float4* __restrict__ dW_gu, float4* __restrict__ dW_d, size_t gu_vec4,
+                                                            size_t d_vec4) {
+  const int n = *n_wchunks;
+  const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int ci = 0; ci < n; ++ci) {
+    const int we = wchunk_expert[ci];
+    if (!(we & WCHUNK_SPLIT)) continue;
+    const int e = we & ~WCHUNK_SPLIT;
+    if (wchunk_row0[ci] != pad_offsets[e]) continue;   // once per expert: at its first chunk
+    float4* gu = dW_gu + (size_t)e * gu_vec4;
+    float4* dd = dW_d + (size_t)e * d_vec4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < gu_vec4; i += (size_t)gridDim.x * blockDim.x) gu[i] = z;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < d_vec4; i += (size_t)gridDim.x * blockDim.x) dd[i] = z;
+  }
+}
+
+cudaError_t launch_zero_split_dw(grouter_ctx* ctx, float* dW_gu, float* dW_d, cudaStream_t st) {
+  const grouter_dims& dm = ctx->dims;
+  const size_t per_gu = (size_t)2 * dm.ffn * dm.d / 4, per_d = (size_t)dm.d * dm.ffn / 4;   // d, ffn multiples of 8
+  zero_split_dw_kernel<<<ctx->num_sms * 4, 256, 0, st>>>(ctx->pp.n_wchunks, ctx->pp.wchunk_expert, ctx->pp.wchunk_row0, ctx->pp.pad_offsets,
+                                                         reinterpret_cast<float4*>(dW_gu), reinterpret_cast<float4*>(dW_d), per_gu, per_d);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,

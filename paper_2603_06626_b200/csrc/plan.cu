@@ -60,7 +60,7 @@ template <typename IdxT>
 __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
                                                                  int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
                                                                  int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
-  extern __shared__ int32_t sm[];  // max(PLAN_WARPS*E, 4*E+4) ints
+  extern __shared__ int32_t sm[];  // max(PLAN_WARPS*E, 5*E+5) ints
   __shared__ int s_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   int32_t* s_off = sm + E_tgt;            // [E+1]
   int32_t* s_pad = sm + 2 * E_tgt + 1;    // [E+1]
   int32_t* s_pair = sm + 3 * E_tgt + 2;   // [E+1] exclusive prefix of 256-row tiles per expert
+  int32_t* s_wch = sm + 4 * E_tgt + 3;    // [E+1] exclusive prefix of weight-gradient row chunks per expert
   __syncthreads();
   for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
     int carry = 0;
@@ -109,39 +110,47 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   if (warp == 0) {
     const int per = (E_tgt + 31) / 32;
     const int e0 = min(lane * per, E_tgt), e1 = min(e0 + per, E_tgt);
-    int sum = 0, psum = 0, tsum = 0;
+    constexpr int CHUNK_BLOCKS = WGRAD_KCHUNK / ROW_TILE;
+    auto chunks_of = [](int blocks) { return blocks == 0 ? 1 : (blocks + CHUNK_BLOCKS - 1) / CHUNK_BLOCKS; };
+    int sum = 0, psum = 0, tsum = 0, wsum = 0;
     for (int e = e0; e < e1; ++e) {
       const int blocks = (s_cnt[e] + ROW_TILE - 1) / ROW_TILE;
       sum += s_cnt[e];
       psum += blocks * ROW_TILE;
       tsum += (blocks + 1) >> 1;
+      wsum += chunks_of(blocks);
     }
-    int isum = sum, ipsum = psum, itsum = tsum;
+    int isum = sum, ipsum = psum, itsum = tsum, iwsum = wsum;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int a = __shfl_up_sync(0xffffffffu, isum, o);
       const int b = __shfl_up_sync(0xffffffffu, ipsum, o);
       const int c = __shfl_up_sync(0xffffffffu, itsum, o);
+      const int w = __shfl_up_sync(0xffffffffu, iwsum, o);
       if (lane >= o) {
         isum += a;
         ipsum += b;
         itsum += c;
+        iwsum += w;
       }
     }
-    int off = isum - sum, poff = ipsum - psum, toff = itsum - tsum;
+    int off = isum - sum, poff = ipsum - psum, toff = itsum - tsum, woff = iwsum - wsum;
     for (int e = e0; e < e1; ++e) {
       const int blocks = (s_cnt[e] + ROW_TILE - 1) / ROW_TILE;
       s_off[e] = off;
       s_pad[e] = poff;
       s_pair[e] = toff;
+      s_wch[e] = woff;
       off += s_cnt[e];
       poff += blocks * ROW_TILE;
       toff += (blocks + 1) >> 1;
+      woff += chunks_of(blocks);
     }
     if (lane == 31) {
       s_off[E_tgt] = isum;
       s_pad[E_tgt] = ipsum;
       s_pair[E_tgt] = itsum;
+      s_wch[E_tgt] = iwsum;
     }
   }
   __syncthreads();
@@ -169,6 +178,19 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
     const int row0 = s_pad[lo] + (t - s_pair[lo]) * 2 * ROW_TILE;
     pp.pair_row0[t] = row0;
     pp.pair_expert[t] = lo | (row0 + ROW_TILE < s_pad[lo + 1] ? PAIR_VALID2 : 0);
+  }
+  // row chunks of the weight-gradient GEMMs: an expert without slots keeps one empty chunk (its gradient is zero-filled)
+  if (tid == 0) *pp.n_wchunks = s_wch[E_tgt];
+  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+    const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
+    const int n = s_wch[e + 1] - s_wch[e];
+    const int base = blocks / n, rem = blocks - base * n;   // chunks of near-equal size: the first `rem` hold one block more
+    for (int c = 0; c < n; ++c) {
+      const int i = s_wch[e] + c;
+      pp.wchunk_expert[i] = e | (n > 1 ? WCHUNK_SPLIT : 0);
+      pp.wchunk_row0[i] = s_pad[e] + (c * base + min(c, rem)) * ROW_TILE;
+      pp.wchunk_rows[i] = (base + (c < rem ? 1 : 0)) * ROW_TILE;
+    }
   }
   // pad rows carry no slot
   for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
@@ -232,7 +254,7 @@ static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, c
   const int R = (int)ctx->R, E = dm.E_tgt;
   const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
   if (phase == 0) {
-    const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 4 * E + 4) ? PLAN_WARPS * E : 4 * E + 4);
+    const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 5 * E + 5) ? PLAN_WARPS * E : 5 * E + 5);
     plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
   } else {
     const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
@@ -282,7 +304,12 @@ constexpr int NA_TICKET = NA_N_TILES + 64;                            // [1]
 constexpr int NA_STATUS = NA_TICKET + 64;                             // [1] used when the caller passes no status word
 constexpr int NA_PAIR_ROW0 = NA_STATUS + 64;                          // [rows/128]
 constexpr int NA_PAIR_EXPERT = NA_PAIR_ROW0 + NOALLOC_MAX_ROWS / ROW_TILE;     // [rows/128]
-constexpr int NA_SLOT_TO_PROW = NA_PAIR_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE;  // [R]
+constexpr int NOALLOC_MAX_WCHUNKS = (NOALLOC_MAX_E + NOALLOC_MAX_ROWS / WGRAD_KCHUNK + 1 + 63) / 64 * 64;
+constexpr int NA_WCHUNK_EXPERT = NA_PAIR_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE; // [chunks]
+constexpr int NA_WCHUNK_ROW0 = NA_WCHUNK_EXPERT + NOALLOC_MAX_WCHUNKS;         // [chunks]
+constexpr int NA_WCHUNK_ROWS = NA_WCHUNK_ROW0 + NOALLOC_MAX_WCHUNKS;           // [chunks]
+constexpr int NA_N_WCHUNKS = NA_WCHUNK_ROWS + NOALLOC_MAX_WCHUNKS;             // [1]
+constexpr int NA_SLOT_TO_PROW = NA_N_WCHUNKS + 64;                             // [R]
 constexpr int NA_PROW_TO_SLOT = NA_SLOT_TO_PROW + NOALLOC_MAX_R;      // [rows]
 constexpr int NA_BLK_PREFIX = NA_PROW_TO_SLOT + NOALLOC_MAX_ROWS;     // [E * blocks]
 constexpr int NA_WORDS = NA_BLK_PREFIX + NOALLOC_MAX_E * NOALLOC_MAX_BLOCKS;
@@ -352,6 +379,10 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.pp.status = status ? status : base + NA_STATUS;
   c.pp.pair_row0 = base + NA_PAIR_ROW0;
   c.pp.pair_expert = base + NA_PAIR_EXPERT;
+  c.pp.wchunk_expert = base + NA_WCHUNK_EXPERT;
+  c.pp.wchunk_row0 = base + NA_WCHUNK_ROW0;
+  c.pp.wchunk_rows = base + NA_WCHUNK_ROWS;
+  c.pp.n_wchunks = base + NA_N_WCHUNKS;
   c.pp.slot_to_prow = base + NA_SLOT_TO_PROW;
   c.pp.prow_to_slot = base + NA_PROW_TO_SLOT;
   c.pp.blk_prefix = base + NA_BLK_PREFIX;

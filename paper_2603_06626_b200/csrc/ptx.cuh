@@ -115,6 +115,14 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t sme
                "r"(smem_src), "r"(x), "r"(y), "r"(z)
                : "memory");
 }
+// Tile reduction shared -> global: every element of the tile is added to the element in global memory (the
+// element type, f32 here, comes from the tensor map); out-of-bounds parts are clipped like a store.
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* tm, uint32_t smem_src, int32_t x, int32_t y, int32_t z) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
+                   reinterpret_cast<uint64_t>(tm)),
+               "r"(smem_src), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // the shared-memory sources of all committed groups have been read
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
