@@ -77,7 +77,7 @@ void grouter_destroy(grouter_ctx* ctx);
  * so it must not be touched in between.  Rows are padded per expert to a
  * multiple of 128, so it is sized for T*k + 128*E_tgt rows.  0 on bad dims. */
 size_t grouter_workspace_bytes(const grouter_dims* dims);
-/* Extra bytes grouter_moe_step_host needs after the workspace proper. */
+/* Extra bytes grouter_moe_step_host needs after the workspace proper (two staging sets). */
 size_t grouter_host_staging_bytes(const grouter_dims* dims);
 
 /* Routing-plan build: a stable counting sort of the R slots by target expert.
@@ -153,16 +153,24 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
                     const void* W_d, void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace,
                     void* stream);
 
-/* One whole step from HOST buffers: copies idx, gates, X, dY to the device
- * (cudaMemcpyAsync on `stream`; pass pinned memory for real overlap), runs plan,
- * fwd and bwd, and copies Y, dX, dgates back.  Weights, weight gradients and
- * fold_map stay on the device.  `workspace` must hold
- * grouter_workspace_bytes + grouter_host_staging_bytes.  Returns after
- * enqueueing; synchronise the stream before reading the host outputs. */
+/* One whole step from HOST buffers: uploads idx, gates, X, dY, runs plan, fwd and bwd on `stream`, and downloads
+ * Y, dX, dgates.  Weights, weight gradients and fold_map stay on the device.  The copies run on two streams the
+ * context owns, ordered against the compute with events: dY is uploaded while plan and fwd run, Y is downloaded
+ * while bwd runs, and with two device staging sets the uploads of step i+1 and the downloads of step i overlap
+ * the compute of their neighbours.  Pass pinned host memory, otherwise the copies serialise.
+ *   workspace: grouter_workspace_bytes + grouter_host_staging_bytes (the latter holds both staging sets).
+ * The call returns after enqueueing.  Host outputs of a step may be read, and its host inputs overwritten,
+ * only after grouter_host_wait says the step is complete; synchronising `stream` alone is NOT enough (the
+ * downloads run on the context's own stream).  Keeping one step in flight therefore needs two sets of host
+ * buffers, used alternately. */
 int grouter_moe_step_host(grouter_ctx* ctx, const void* idx_host, const void* gates_host, const void* X_host,
                           const void* dY_host, const int32_t* fold_map, const void* W_gu, const void* W_d,
                           void* Y_host, void* dX_host, float* dgates_host, float* dW_gu, float* dW_d,
                           void* workspace, void* stream);
+/* Blocks the calling host thread until all but the `steps_in_flight` (0 or 1) most recently submitted
+ * grouter_moe_step_host calls are complete: their host outputs are written and their host inputs consumed.
+ * (No counterpart in the paper: host-side plumbing of the step call.) */
+int grouter_host_wait(grouter_ctx* ctx, int32_t steps_in_flight);
 
 /* Synchronises `stream` and returns the sticky device status (GROUTER_OK,
  * GROUTER_ERR_BAD_INDEX, GROUTER_ERR_TIMEOUT) or GROUTER_ERR_CUDA; clears it. */

@@ -19,7 +19,7 @@ GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
-           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc"]
+           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW"]
 
@@ -66,6 +66,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_moe_bwd.restype = ctypes.c_int
     lib.grouter_moe_step_host.argtypes = [vp] * 15
     lib.grouter_moe_step_host.restype = ctypes.c_int
+    lib.grouter_host_wait.argtypes = [vp, ctypes.c_int32]
+    lib.grouter_host_wait.restype = ctypes.c_int
     lib.grouter_status.argtypes = [vp, vp]
     lib.grouter_status.restype = ctypes.c_int
     lib.grouter_strerror.argtypes = [ctypes.c_int]
@@ -164,8 +166,13 @@ class GrouterLayer:
                                         _ptr(dW_d), _ptr(dgates), _ptr(self.workspace), _stream()), "grouter_moe_bwd")
         return dX, dW_gu, dW_d, dgates
 
+    def host_wait(self, steps_in_flight: int = 0) -> None:
+        """Blocks until all but the `steps_in_flight` (0 or 1) most recent step_host calls are complete."""
+        _check(self.lib.grouter_host_wait(self.ctx, steps_in_flight), "grouter_host_wait")
+
     def step_host(self, idx_h, gates_h, X_h, dY_h, fold_map, W_gu, W_d, Y_h, dX_h, dgates_h, dW_gu, dW_d):
-        """Whole step from pinned host tensors (idx, gates, X, dY in; Y, dX, dgates out)."""
+        """Whole step from pinned host tensors (idx, gates, X, dY in; Y, dX, dgates out).  Asynchronous: read the
+        outputs (and reuse the inputs) only after host_wait() reports the step complete."""
         _check(self.lib.grouter_moe_step_host(self.ctx, _ptr(idx_h), _ptr(gates_h), _ptr(X_h), _ptr(dY_h), _ptr(fold_map), _ptr(W_gu),
                                               _ptr(W_d), _ptr(Y_h), _ptr(dX_h), _ptr(dgates_h), _ptr(dW_gu), _ptr(dW_d),
                                               _ptr(self.workspace), _stream()), "grouter_moe_step_host")

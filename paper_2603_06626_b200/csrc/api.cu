@@ -132,7 +132,7 @@ size_t grouter_workspace_bytes(const grouter_dims* dims) {
 
 size_t grouter_host_staging_bytes(const grouter_dims* dims) {
   if (check_dims(dims) != GROUTER_OK) return 0;
-  return staging_layout(*dims).bytes;
+  return 2 * staging_layout(*dims).bytes;   // two sets: consecutive steps are in flight together
 }
 
 int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
@@ -160,6 +160,23 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->ev_start = c->ev_stop = nullptr;
   c->ev_slot = nullptr;
   c->ev_cap = c->ev_used = 0;
+  c->host_steps = 0;
+  c->s_in = c->s_out = nullptr;
+  for (int i = 0; i < 2; ++i) c->ev_in_fwd[i] = c->ev_in_bwd[i] = c->ev_fwd_done[i] = c->ev_bwd_done[i] = c->ev_out_done[i] = nullptr;
+  {
+    bool ok = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&c->ev_in_fwd[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_in_bwd[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_fwd_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_bwd_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&c->ev_out_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      grouter_destroy(c);
+      return GROUTER_ERR_CUDA;
+    }
+  }
   const int E = dims->E_tgt;
   size_t off = 0;
   auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
@@ -168,12 +185,12 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   const size_t o_we = take((size_t)c->max_wchunks * 4), o_wr = take((size_t)c->max_wchunks * 4), o_wn = take((size_t)c->max_wchunks * 4), o_nw = take(4);
   const size_t o_p2s = take((size_t)c->R_pad_max * 4), o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
   if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
-    delete c;
+    c->d_block = nullptr;
+    grouter_destroy(c);
     return GROUTER_ERR_CUDA;
   }
   if (cudaMemset(c->d_block, 0, off) != cudaSuccess) {
-    cudaFree(c->d_block);
-    delete c;
+    grouter_destroy(c);
     return GROUTER_ERR_CUDA;
   }
   char* b = static_cast<char*>(c->d_block);
@@ -199,6 +216,13 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
 void grouter_destroy(grouter_ctx* ctx) {
   if (!ctx) return;
   free_events(ctx);
+  if (ctx->s_in) cudaStreamDestroy(ctx->s_in);
+  if (ctx->s_out) cudaStreamDestroy(ctx->s_out);
+  for (int i = 0; i < 2; ++i) {
+    cudaEvent_t evs[5] = {ctx->ev_in_fwd[i], ctx->ev_in_bwd[i], ctx->ev_fwd_done[i], ctx->ev_bwd_done[i], ctx->ev_out_done[i]};
+    for (cudaEvent_t e : evs)
+      if (e) cudaEventDestroy(e);
+  }
   if (ctx->d_block) cudaFree(ctx->d_block);
   delete ctx;
 }
@@ -301,24 +325,52 @@ int grouter_moe_step_host(grouter_ctx* ctx, const void* idx_host, const void* ga
   const grouter_dims& dm = ctx->dims;
   const size_t ws_bytes = carve_workspace(dm, ctx->R_pad_max, nullptr).bytes;
   const Staging sg = staging_layout(dm);
-  char* sb = static_cast<char*>(workspace) + ws_bytes;
+  const int set = (int)(ctx->host_steps & 1);
+  char* sb = static_cast<char*>(workspace) + ws_bytes + (size_t)set * sg.bytes;
   const size_t R = (size_t)dm.T * dm.k, Td = (size_t)dm.T * dm.d;
   const size_t idx_b = R * (dm.idx_dtype == GROUTER_IDX_U8 ? 1 : 4), gate_b = R * (dm.gate_dtype == GROUTER_GATE_BF16 ? 2 : 4);
-  if (cudaMemcpyAsync(sb + sg.idx, idx_host, idx_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (cudaMemcpyAsync(sb + sg.gates, gates_host, gate_b, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (cudaMemcpyAsync(sb + sg.X, X_host, Td * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (cudaMemcpyAsync(sb + sg.dY, dY_host, Td * 2, cudaMemcpyHostToDevice, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+
+  // uploads (copy stream): the staging set is free once the step that used it last has downloaded its results
+  if (!ok(cudaStreamWaitEvent(ctx->s_in, ctx->ev_out_done[set], 0))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(sb + sg.idx, idx_host, idx_b, cudaMemcpyHostToDevice, ctx->s_in))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(sb + sg.gates, gates_host, gate_b, cudaMemcpyHostToDevice, ctx->s_in))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(sb + sg.X, X_host, Td * 2, cudaMemcpyHostToDevice, ctx->s_in))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaEventRecord(ctx->ev_in_fwd[set], ctx->s_in))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(sb + sg.dY, dY_host, Td * 2, cudaMemcpyHostToDevice, ctx->s_in))) return GROUTER_ERR_CUDA;   // during plan + fwd
+  if (!ok(cudaEventRecord(ctx->ev_in_bwd[set], ctx->s_in))) return GROUTER_ERR_CUDA;
+
+  // compute (caller's stream)
+  if (!ok(cudaStreamWaitEvent(st, ctx->ev_in_fwd[set], 0))) return GROUTER_ERR_CUDA;
   int rc = grouter_plan(ctx, sb + sg.idx, fold_map, reinterpret_cast<int32_t*>(sb + sg.counts), reinterpret_cast<int32_t*>(sb + sg.offsets),
                         reinterpret_cast<int32_t*>(sb + sg.r2s), reinterpret_cast<int32_t*>(sb + sg.s2r), stream);
   if (rc != GROUTER_OK) return rc;
   rc = grouter_moe_fwd(ctx, sb + sg.X, sb + sg.gates, W_gu, W_d, sb + sg.Y, workspace, stream);
   if (rc != GROUTER_OK) return rc;
+  if (!ok(cudaEventRecord(ctx->ev_fwd_done[set], st))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaStreamWaitEvent(st, ctx->ev_in_bwd[set], 0))) return GROUTER_ERR_CUDA;
   rc = grouter_moe_bwd(ctx, sb + sg.dY, sb + sg.X, sb + sg.gates, W_gu, W_d, sb + sg.dX, dW_gu, dW_d,
                        reinterpret_cast<float*>(sb + sg.dgates), workspace, stream);
   if (rc != GROUTER_OK) return rc;
-  if (cudaMemcpyAsync(Y_host, sb + sg.Y, Td * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (cudaMemcpyAsync(dX_host, sb + sg.dX, Td * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  if (cudaMemcpyAsync(dgates_host, sb + sg.dgates, R * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (!ok(cudaEventRecord(ctx->ev_bwd_done[set], st))) return GROUTER_ERR_CUDA;
+
+  // downloads (copy stream): Y leaves while the backward pass runs
+  if (!ok(cudaStreamWaitEvent(ctx->s_out, ctx->ev_fwd_done[set], 0))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(Y_host, sb + sg.Y, Td * 2, cudaMemcpyDeviceToHost, ctx->s_out))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaStreamWaitEvent(ctx->s_out, ctx->ev_bwd_done[set], 0))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(dX_host, sb + sg.dX, Td * 2, cudaMemcpyDeviceToHost, ctx->s_out))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(dgates_host, sb + sg.dgates, R * 4, cudaMemcpyDeviceToHost, ctx->s_out))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaEventRecord(ctx->ev_out_done[set], ctx->s_out))) return GROUTER_ERR_CUDA;
+  ctx->host_steps += 1;
+  return GROUTER_OK;
+}
+
+int grouter_host_wait(grouter_ctx* ctx, int32_t steps_in_flight) {
+  if (!ctx || steps_in_flight < 0 || steps_in_flight > 1) return GROUTER_ERR_INVALID_ARG;
+  // step i records ev_out_done[i & 1] last; waiting for it covers every earlier step as well (one download stream)
+  const int64_t last_needed = ctx->host_steps - 1 - steps_in_flight;
+  if (last_needed < 0) return GROUTER_OK;
+  if (cudaEventSynchronize(ctx->ev_out_done[last_needed & 1]) != cudaSuccess) return GROUTER_ERR_CUDA;
   return GROUTER_OK;
 }
 

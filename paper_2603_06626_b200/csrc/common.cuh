@@ -78,6 +78,10 @@ struct grouter_ctx {
   bool planned;
   bool forwarded;
   int num_sms;
+  // copy pipeline of grouter_moe_step_host: uploads, compute and downloads of consecutive steps overlap
+  cudaStream_t s_in, s_out;          // host->device and device->host copy streams
+  cudaEvent_t ev_in_fwd[2], ev_in_bwd[2], ev_fwd_done[2], ev_bwd_done[2], ev_out_done[2];   // per staging set
+  int64_t host_steps;                // steps submitted so far; step i uses staging set i & 1
   // optional per-kernel timing (event pool)
   cudaEvent_t* ev_start;
   cudaEvent_t* ev_stop;
