@@ -41,6 +41,58 @@ MOVER_SLOTS = ["gather_X", "combine_Y", "gather_dY", "reduce_dX"]
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+def kernel_source_tag() -> str:
+    """Short hash of the CUDA sources: DRAM counters taken with another build are not reported."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2603_06626_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()[:12]
+
+
+def recorded_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
+    profiles/dram_traffic.txt, or None when there is no capture of this kernel on this workload with this build."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    tag = kernel_source_tag()
+    for line in open(path):
+        parts = line.split()
+        if len(parts) >= 4 and not line.startswith("#") and parts[0] == workload and parts[1] == kernel and parts[3] == tag:
+            return float(parts[2])
+    return None
+
+
+def plan_at_scale(dev, T=1 << 22, k=8, E=128, iters=5):
+    """The plan build at a size where bytes, not launch latency, decide its time: uniform ids, T*k = 2^25 slots.
+    Algorithmic bytes: ids read twice (histogram pass, permutation pass) and the two permutations written."""
+    import torch
+    from paper_2603_06626_b200 import binding
+    layer = binding.GrouterLayer(T, 8, 8, E, k, device=str(dev))
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    idx = torch.randint(0, E, (T, k), dtype=torch.uint8, device=dev, generator=g)
+    for _ in range(2):
+        layer.plan(idx)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        layer.plan(idx)
+    e1.record()
+    torch.cuda.synchronize()
+    layer.check_status()
+    ms = e0.elapsed_time(e1) / iters
+    R = T * k
+    assert int(layer.counts.sum().item()) == R
+    layer.close()
+    by = 2.0 * R + 2.0 * R * 4
+    return {"T": T, "k": k, "E": E, "ms": ms, "algorithmic_bytes": by, "gbs": by / (ms * 1e-3) / 1e9}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -201,6 +253,7 @@ def main():
     ap.add_argument("--cpu-baseline-tokens", type=int, default=48)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-plan-scale", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -342,11 +395,9 @@ def main():
             ent["frac_of_hbm"] = ent["gbs"] / peaks["hbm_gbs"]
         kernels[name] = ent
     dom = max(GEMM_SLOTS, key=lambda k: per_kernel[k][0])
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            traffic = json.load(f).get(w.name, {}).get(dom)
+    traffic = recorded_traffic(w.name, dom)
+    for name, ent in kernels.items():
+        ent["traffic"] = recorded_traffic(w.name, name)
     roofline = {"kernel": dom, "bound": "tensor", "achieved": kernels[dom]["tflops"], "peak": peaks["bf16_tflops_sustained"],
                 "unit": "TFLOP/s", "frac": kernels[dom]["tflops"] / peaks["bf16_tflops_sustained"], "traffic": traffic,
                 "peak_source": f"{peak_src} cuBLAS bf16, sustained (kernel timed inside a long step); burst peak "
@@ -366,6 +417,11 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if world == 1 and not args.no_plan_scale:
+        layer.close()
+        ps = plan_at_scale(dev)
+        ps["frac_of_hbm"] = ps["gbs"] / peaks["hbm_gbs"]
+        line["plan_scaled"] = ps
     if world == 1 and not args.no_cpu_baseline:
         v, dt, threads = oracle_sample_tokens_per_sec(w, li, args.cpu_baseline_tokens)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
