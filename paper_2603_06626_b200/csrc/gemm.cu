@@ -237,6 +237,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   volatile int* abort_flag = &s_abort;
 
   const int n_tiles = total_tiles<MODE>(p);
+  // L2 residency: B (an expert's weights, or the row chunk every output tile of a weight gradient reads) is
+  // reused by other CTA pairs and later tiles; the outputs are streamed out once and must not displace it.
+  const uint64_t keep_a = ptx::l2_policy_evict_normal(), keep_b = ptx::l2_policy_evict_last(), stream_out = ptx::l2_policy_evict_first();
 
   if (warp == 0) {
     // ===================== TMA producer (both CTAs) =====================
@@ -253,18 +256,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t fb = ptx::map_to_cta(full_bar(s), 0);   // both CTAs' bytes complete on the leader's barrier
           const int k0 = ks * BK;
           if (!A_MN) {
-            ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y);                       // box {64 k, 128 rows}
+            ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y, keep_a);                       // box {64 k, 128 rows}
           } else {
             const int ay = (MODE == MODE_DENSE ? 0 : ti.a_y) + k0;
-            ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay);                       // 2 x box {64 m, 64 k}
-            ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay);
+            ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay, keep_a);                       // 2 x box {64 m, 64 k}
+            ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay, keep_a);
           }
           if (!B_MN) {
-            ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y);                       // box {64 k, 128 rows}
+            ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y, keep_b);                       // box {64 k, 128 rows}
           } else {
             const int by = (MODE == MODE_DENSE ? 0 : ti.b_y) + k0;
-            ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by);                       // 2 x box {64 n, 64 k}
-            ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by);
+            ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by, keep_b);                       // 2 x box {64 n, 64 k}
+            ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by, keep_b);
           }
           if (++s == STAGES) {
             s = 0;
@@ -369,7 +372,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       ptx::fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        ptx::tma_store_2d(tm, blk, x, y);
+        ptx::tma_store_2d(tm, blk, x, y, stream_out);
         ptx::bulk_commit();
       }
     };
@@ -378,7 +381,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       __syncwarp();
       if (lane == 0) {
         if (add) ptx::tma_reduce_add_3d(tm, blk, x, y, z);
-        else ptx::tma_store_3d(tm, blk, x, y, z);
+        else ptx::tma_store_3d(tm, blk, x, y, z, stream_out);
         ptx::bulk_commit();
       }
     };
