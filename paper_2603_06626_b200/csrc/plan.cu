@@ -2,8 +2,8 @@
 // expert, in two launches.
 //
 //   plan_hist_kernel    every block histograms a contiguous chunk of slots
-//                       (one private histogram per warp, built with
-//                       __match_any_sync so no atomics are needed); the last
+//                       (one private histogram per warp, built from warp
+//                       ballots so no atomics are needed); the last
 //                       block to finish turns the per-block histograms into
 //                       exclusive prefixes over blocks, scans the expert
 //                       counts into offsets, and lays out the 128-row-padded
@@ -19,10 +19,8 @@
 
 namespace grouter {
 
-template <typename IdxT>
-__device__ __forceinline__ int load_expert(const IdxT* __restrict__ idx, int s, const int32_t* __restrict__ fold_map, int E_src,
-                                           int E_tgt, int32_t* status) {
-  int raw = (int)idx[s];
+// Target expert of a raw id: range check, fold map, range check; a bad id or fold target counts as expert 0.
+__device__ __forceinline__ int fold_expert(int raw, const int32_t* __restrict__ fold_map, int E_src, int E_tgt, int32_t* status) {
   bool bad = false;
   if ((unsigned)raw >= (unsigned)E_src) {
     bad = true;
@@ -37,6 +35,19 @@ __device__ __forceinline__ int load_expert(const IdxT* __restrict__ idx, int s, 
   return e;
 }
 
+// Lanes of the warp that hold the same key as this lane (invalid lanes carry key -1 and match each other only).
+// One ballot per key bit: constant cost, unlike match.any whose cost grows with the number of distinct keys.
+__device__ __forceinline__ unsigned same_key_lanes(int key, int key_bits) {
+  unsigned peers = __ballot_sync(0xffffffffu, key >= 0);
+  if (key < 0) peers = ~peers;
+  for (int b = 0; b < key_bits; ++b) {
+    const unsigned ones = __ballot_sync(0xffffffffu, (key >> b) & 1);
+    peers &= ((key >> b) & 1) ? ones : ~ones;
+  }
+  return peers;
+}
+__device__ __forceinline__ int bits_for(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
+
 // Per-warp histograms of this block's chunk into hist[w*E + e] (smem, pre-zeroed).
 template <typename IdxT>
 __device__ __forceinline__ void warp_histogram(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map, int R, int E_src,
@@ -45,11 +56,15 @@ __device__ __forceinline__ void warp_histogram(const IdxT* __restrict__ idx, con
   const int wlen = chunk / PLAN_WARPS;
   const int base = blockIdx.x * chunk + warp * wlen;
   int32_t* h = hist + warp * E_tgt;
+  const int key_bits = bits_for(E_tgt);
+  int raw_next = (base + lane < R) ? (int)idx[base + lane] : 0;   // ids are fetched one iteration ahead
   for (int i = 0; i < wlen; i += 32) {
     const int s = base + i + lane;
     const bool valid = s < R;
-    const int e = valid ? load_expert(idx, s, fold_map, E_src, E_tgt, status) : -1;
-    const unsigned mask = __match_any_sync(0xffffffffu, e);
+    const int raw = raw_next;
+    if (i + 32 < wlen && s + 32 < R) raw_next = (int)idx[s + 32];
+    const int e = valid ? fold_expert(raw, fold_map, E_src, E_tgt, status) : -1;
+    const unsigned mask = same_key_lanes(e, key_bits);
     if (valid && lane == __ffs(mask) - 1) h[e] += __popc(mask);
     __syncwarp();
     if (base + i + 32 >= R) break;
@@ -90,21 +105,44 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   int32_t* s_pair = sm + 3 * E_tgt + 2;   // [E+1] exclusive prefix of 256-row tiles per expert
   int32_t* s_wch = sm + 4 * E_tgt + 3;    // [E+1] exclusive prefix of weight-gradient row chunks per expert
   __syncthreads();
-  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
-    int carry = 0;
-    for (int b0 = 0; b0 < nblk; b0 += 32) {
-      const int b = b0 + lane;
-      const int v = b < nblk ? __ldcg(pp.blk_prefix + e * nblk + b) : 0;
-      int incl = v;
+  // Exclusive prefix over blocks of every expert's per-block counts (row e of blk_prefix), and the expert totals.
+  // Eight lanes share one expert: each sums a contiguous segment of the row with its loads batched eight deep, the
+  // eight segment sums are scanned with shuffles, and a second sweep writes the running prefixes back.
+  {
+    const int grp = lane >> 3, gl = lane & 7;
+    const int seg = (nblk + 7) >> 3;
+    for (int e0 = warp * 4; e0 < E_tgt; e0 += PLAN_WARPS * 4) {
+      const int e = e0 + grp;
+      const bool have = e < E_tgt;
+      int32_t* rowp = pp.blk_prefix + (size_t)(have ? e : 0) * nblk;
+      const int b_lo = min(gl * seg, nblk), b_hi = have ? min(b_lo + seg, nblk) : b_lo;
+      int sum = 0;
+      for (int b = b_lo; b < b_hi; b += 8) {
+        int v[8];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += n;
+        for (int j = 0; j < 8; ++j) v[j] = (b + j < b_hi) ? __ldcg(rowp + b + j) : 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sum += v[j];
       }
-      if (b < nblk) pp.blk_prefix[e * nblk + b] = carry + incl - v;
-      carry += __shfl_sync(0xffffffffu, incl, 31);
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, o, 8);
+        if (gl >= o) incl += n;
+      }
+      int run = incl - sum;
+      for (int b = b_lo; b < b_hi; b += 8) {
+        int v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (b + j < b_hi) ? __ldcg(rowp + b + j) : 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (b + j < b_hi) rowp[b + j] = run;
+          run += v[j];
+        }
+      }
+      if (have && gl == 7) s_cnt[e] = incl;
     }
-    if (lane == 0) s_cnt[e] = carry;
   }
   __syncthreads();
   if (warp == 0) {
@@ -227,11 +265,15 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_permute_kernel(const IdxT* 
   const int base = blockIdx.x * chunk + warp * wlen;
   int32_t* cur = sm + warp * E_tgt;
   const unsigned lt = (1u << lane) - 1u;
+  const int key_bits = bits_for(E_tgt);
+  int raw_next = (base + lane < R) ? (int)idx[base + lane] : 0;   // ids are fetched one iteration ahead
   for (int i = 0; i < wlen; i += 32) {
     const int s = base + i + lane;
     const bool valid = s < R;
-    const int e = valid ? load_expert(idx, s, fold_map, E_src, E_tgt, pp.status) : -1;
-    const unsigned mask = __match_any_sync(0xffffffffu, e);
+    const int raw = raw_next;
+    if (i + 32 < wlen && s + 32 < R) raw_next = (int)idx[s + 32];
+    const int e = valid ? fold_expert(raw, fold_map, E_src, E_tgt, pp.status) : -1;
+    const unsigned mask = same_key_lanes(e, key_bits);
     const int row = valid ? cur[e] + __popc(mask & lt) : 0;
     __syncwarp();
     if (valid && lane == 31 - __clz(mask)) cur[e] = row + 1;
