@@ -22,7 +22,8 @@
  *     range, a bounded wait that ran out) set a sticky status word; the
  *     kernels keep every access in bounds and finish, and grouter_status()
  *     reports it.  Nothing traps.
- *   - Outputs are overwritten, never accumulated into.
+ *   - Outputs are overwritten, never accumulated into (dW_* excepted under
+ *     GROUTER_FLAG_ACCUMULATE_DW).
  *
  * Sizes: T tokens, d model width, ffn expert hidden width, k experts per token,
  * E_src ids that may appear in idx, E_tgt experts that own weights
@@ -54,6 +55,9 @@ enum {
 
 enum { GROUTER_IDX_U8 = 0, GROUTER_IDX_I32 = 1 };
 enum { GROUTER_GATE_BF16 = 0, GROUTER_GATE_F32 = 1 };
+/* grouter_moe_bwd adds the weight gradients into dW_gu / dW_d instead of overwriting them (gradient accumulation
+ * over micro-batches; the caller zeroes them before the first one).  Experts without slots are left untouched. */
+enum { GROUTER_FLAG_ACCUMULATE_DW = 1 };
 
 typedef struct grouter_ctx grouter_ctx; /* opaque */
 
@@ -61,7 +65,7 @@ typedef struct {
   int32_t T, d, ffn, E_src, E_tgt, k;
   int32_t idx_dtype;  /* GROUTER_IDX_U8 (the paper's cache format, E_src <= 256) or GROUTER_IDX_I32 */
   int32_t gate_dtype; /* GROUTER_GATE_BF16 (the paper's cache format) or GROUTER_GATE_F32           */
-  int32_t flags;      /* reserved, pass 0 */
+  int32_t flags;      /* 0 or an OR of GROUTER_FLAG_* */
 } grouter_dims;
 
 /* Creates a context for one layer shape on the current CUDA device.  Host call;
@@ -145,7 +149,8 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
  *   dY     [T,d] bf16                 dX     [T,d] bf16 out
  *   dW_gu  [E_tgt, 2*ffn, d] f32 out  dW_d   [E_tgt, d, ffn] f32 out
  *   dgates [T,k] f32 out: dgates[t,j] = <dY[t,:], f_{e(t,j)}(X[t,:])> (gates are leaf inputs)
- * Experts that received no slot get exact zeros in dW_*.  An expert with more than 4096 rows is contracted in
+ * Experts that received no slot get exact zeros in dW_* (with GROUTER_FLAG_ACCUMULATE_DW every expert's gradient is
+ * added to what dW_* holds, and such experts are left as they are).  An expert with more than 4096 rows is contracted in
  * chunks of rows that are added into its gradient in no fixed order, so its dW_* may differ in the last bits
  * from run to run; everything else (Y, dX, dgates, dW_* of smaller experts) is bit-reproducible.  Uses the workspace
  * contents left by the matching grouter_moe_fwd (else INVALID_STATE). */

@@ -15,6 +15,7 @@ import torch
 from . import build as _build
 
 IDX_U8, IDX_I32 = 0, 1
+FLAG_ACCUMULATE_DW = 1
 GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
@@ -107,10 +108,10 @@ class GrouterLayer:
     """One layer shape: owns the context and the workspace; thin calls into the C ABI."""
 
     def __init__(self, T: int, d: int, ffn: int, E_src: int, k: int, E_tgt: Optional[int] = None, idx_dtype: int = IDX_U8,
-                 gate_dtype: int = GATE_BF16, device: str = "cuda:0", host_staging: bool = False):
+                 gate_dtype: int = GATE_BF16, device: str = "cuda:0", host_staging: bool = False, flags: int = 0):
         self.lib = load_library()
         self.device = torch.device(device)
-        self.dims = GrouterDims(T, d, ffn, E_src, E_src if E_tgt is None else E_tgt, k, idx_dtype, gate_dtype, 0)
+        self.dims = GrouterDims(T, d, ffn, E_src, E_src if E_tgt is None else E_tgt, k, idx_dtype, gate_dtype, flags)
         self.T, self.d, self.ffn, self.k = T, d, ffn, k
         self.E_src, self.E_tgt = E_src, self.dims.E_tgt
         self.R = T * k

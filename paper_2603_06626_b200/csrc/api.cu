@@ -16,6 +16,7 @@ int check_dims(const grouter_dims* dm) {
   if (dm->T < 1 || dm->d < 1 || dm->ffn < 1 || dm->E_src < 1 || dm->E_tgt < 1 || dm->k < 1) return GROUTER_ERR_INVALID_ARG;
   if (dm->idx_dtype != GROUTER_IDX_U8 && dm->idx_dtype != GROUTER_IDX_I32) return GROUTER_ERR_INVALID_ARG;
   if (dm->gate_dtype != GROUTER_GATE_BF16 && dm->gate_dtype != GROUTER_GATE_F32) return GROUTER_ERR_INVALID_ARG;
+  if (dm->flags & ~GROUTER_FLAG_ACCUMULATE_DW) return GROUTER_ERR_INVALID_ARG;
   if (dm->d % 8 || dm->ffn % 8) return GROUTER_ERR_UNSUPPORTED;
   if (dm->E_tgt > 1024 || dm->k > 32) return GROUTER_ERR_UNSUPPORTED;
   if (dm->idx_dtype == GROUTER_IDX_U8 && dm->E_src > 256) return GROUTER_ERR_UNSUPPORTED;
@@ -293,7 +294,9 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
   }
   {
     Timed tm(ctx, 12, st);
-    if (launch_zero_split_dw(ctx, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    // (when accumulating, the caller's gradients are the starting value of every expert's sum: nothing to zero)
+    if (!(ctx->dims.flags & GROUTER_FLAG_ACCUMULATE_DW) && launch_zero_split_dw(ctx, dW_gu, dW_d, st) != cudaSuccess)
+      return GROUTER_ERR_CUDA;
   }
   {
     Timed tm(ctx, 8, st);

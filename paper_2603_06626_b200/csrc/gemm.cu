@@ -52,6 +52,7 @@ struct GemmParams {
   const int32_t* wchunk_row0;  // device [chunks] first padded row
   const int32_t* wchunk_rows;  // device [chunks] rows, multiple of 128
   int32_t E, d, F;
+  int32_t accumulate;          // weight-gradient modes: add every tile into the caller's gradient
   int32_t M, N, K;             // DENSE: problem; WGRAD: per-expert output M x N
   int32_t tiles_m, tiles_n;    // output tiles per problem (tiles_m unused by row-parallel modes)
   int64_t R_pad_max;
@@ -131,7 +132,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
     const int mt = r / p.tiles_n, nt = r - mt * p.tiles_n;
     const int we = __ldg(p.wchunk_expert + ci);
     ti.e = we & ~WCHUNK_SPLIT;
-    ti.add = (we & WCHUNK_SPLIT) != 0;
+    ti.add = (we & WCHUNK_SPLIT) != 0 || p.accumulate != 0;
     const int k0 = __ldg(p.wchunk_row0 + ci), k1 = k0 + __ldg(p.wchunk_rows + ci);
     ti.row0 = mt * PM + rank * BM;
     ti.col0 = nt * BN;
@@ -526,7 +527,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + (size_t)ti.row0 + r] = dgate;
         }
       } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile, four 32-column blocks per warp
-        if (y0 < ti.row0 + ti.m_valid) {
+        // (an expert without rows has nothing to add when accumulating; otherwise its tile is stored as zeros)
+        if (y0 < ti.row0 + ti.m_valid && (have_acc || !ti.add)) {
 #pragma unroll
           for (int blk = 0; blk < 4; ++blk) {
             const int cb = half * 128 + blk * 32;
@@ -662,6 +664,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.d = d;
   p.F = F;
   p.R_pad_max = ctx->R_pad_max;
+  p.accumulate = (dm.flags & GROUTER_FLAG_ACCUMULATE_DW) ? 1 : 0;
   p.prow_to_slot = ctx->pp.prow_to_slot;
   p.gates = gates;
   p.gate_is_f32 = dm.gate_dtype == GROUTER_GATE_F32;

@@ -198,3 +198,44 @@ def test_plan_reuse_across_layers_and_determinism():
     for a, b in zip(r1, r2):
         assert torch.equal(a, b)
     layer.close()
+
+
+def test_accumulate_dw_over_micro_batches():
+    """GROUTER_FLAG_ACCUMULATE_DW: two micro-batches with different routing add up in the caller's zeroed gradients;
+    the sum is checked against the oracle's sum, expert by expert (one expert gets slots in neither batch)."""
+    from paper_2603_06626_b200 import binding
+    base = synth.custom_workload("acc", T=1536, d=256, ffn=384, E=12, k=3, seed=21)
+    route = synth.custom_workload("acc", T=1536, d=256, ffn=384, E=11, k=3, load="zipf", zipf_s=1.2, seed=21)   # ids 0..10: expert 11 idle
+    batches = [synth.make_layer_inputs(synth.reseeded(route, 21 + i), with_weights=False) for i in range(2)]
+    W_gu_bits = np.stack([synth.expert_W_gu(base, e) for e in range(base.E_tgt)])
+    W_d_bits = np.stack([synth.expert_W_d(base, e) for e in range(base.E_tgt)])
+    W_gu, W_d = bits_to_bf16(W_gu_bits), bits_to_bf16(W_d_bits)
+    layer = binding.GrouterLayer(base.T, base.d, base.ffn, base.E_src, base.k, flags=binding.FLAG_ACCUMULATE_DW)
+    dW_gu = torch.zeros(W_gu.shape, dtype=torch.float32, device="cuda:0")
+    dW_d = torch.zeros(W_d.shape, dtype=torch.float32, device="cuda:0")
+    weights = orc.Weights(synth.bf16_bits_to_f64(W_gu_bits), synth.bf16_bits_to_f64(W_d_bits))
+    want_gu = np.zeros(W_gu.shape, dtype=np.float64)
+    want_d = np.zeros(W_d.shape, dtype=np.float64)
+    touched = np.zeros(base.E_tgt, dtype=bool)
+    for li in batches:
+        idx, gates, X, dY = to_dev(li.idx), bits_to_bf16(li.gates), bits_to_bf16(li.X), bits_to_bf16(li.dY)
+        layer.plan(idx)
+        layer.forward(X, gates, W_gu, W_d)
+        layer.backward(dY, X, gates, W_gu, W_d, dW_gu=dW_gu, dW_d=dW_d)
+        touched |= layer.counts.cpu().numpy() > 0
+        f64 = synth.bf16_bits_to_f64
+        _, _, dW = orc.moe_backward(f64(li.dY), f64(li.X), li.idx, f64(li.gates), weights, base.E_tgt)
+        for e in range(base.E_tgt):
+            want_gu[e] += dW[e][0]
+            want_d[e] += dW[e][1]
+    layer.check_status()
+    got_gu, got_d = dW_gu.double().cpu().numpy(), dW_d.double().cpu().numpy()
+    assert not touched[11] and touched[:11].all()
+    for e in range(base.E_tgt):
+        if not touched[e]:
+            assert not got_gu[e].any() and not got_d[e].any()
+        else:
+            assert orc.rel_frobenius(got_gu[e], want_gu[e]) < TOL and orc.rel_frobenius(got_d[e], want_d[e]) < TOL
+    layer.close()
+    with pytest.raises(binding.GrouterError):
+        binding.GrouterLayer(64, 64, 64, 4, 2, flags=4)      # unknown flag bit
