@@ -93,6 +93,43 @@ def plan_at_scale(dev, T=1 << 22, k=8, E=128, iters=5):
     return {"T": T, "k": k, "E": E, "ms": ms, "algorithmic_bytes": by, "gbs": by / (ms * 1e-3) / 1e9}
 
 
+def router_head_leg(dev, T=32768, d_h=512, E_src=128, E_tgt=128, k=8, iters=20):
+    """The step before the plan (Eq. 2): scores of a 512-wide router over 128 experts, top-8, softmax, uint8/bf16 record.
+    Synthetic hidden states and score layer.  Algorithmic bytes: H and W_s read, the 3k-byte record written."""
+    import torch
+    from paper_2603_06626_b200 import binding
+    lib = binding.load_library()
+    g = torch.Generator(device=dev)
+    g.manual_seed(11)
+    H = torch.randn((T, d_h), device=dev, generator=g).to(torch.bfloat16)
+    W = (torch.randn((E_src, d_h), device=dev, generator=g) / d_h ** 0.5).to(torch.bfloat16)
+    idx = torch.empty((T, k), dtype=torch.uint8, device=dev)
+    gates = torch.empty((T, k), dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(lib.grouter_route_workspace_bytes(T, E_src, E_tgt), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        rc = lib.grouter_route(H.data_ptr(), W.data_ptr(), None, T, d_h, E_src, E_tgt, k, binding.NORM_SOFTMAX, idx.data_ptr(),
+                               gates.data_ptr(), None, ws.data_ptr(), status.data_ptr(), st)
+        assert rc == 0, rc
+
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ms = e0.elapsed_time(e1) / iters
+    by = T * d_h * 2.0 + E_src * d_h * 2.0 + 3.0 * k * T
+    return {"T": T, "d_h": d_h, "E": E_src, "k": k, "ms": ms, "tokens_per_s": T / (ms * 1e-3), "algorithmic_bytes": by,
+            "gbs": by / (ms * 1e-3) / 1e9, "gpu_launches_per_call": 3}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -422,6 +459,9 @@ def main():
         ps = plan_at_scale(dev)
         ps["frac_of_hbm"] = ps["gbs"] / peaks["hbm_gbs"]
         line["plan_scaled"] = ps
+        rh = router_head_leg(dev)
+        rh["frac_of_hbm"] = rh["gbs"] / peaks["hbm_gbs"]
+        line["router_head"] = rh
     if world == 1 and not args.no_cpu_baseline:
         v, dt, threads = oracle_sample_tokens_per_sec(w, li, args.cpu_baseline_tokens)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,

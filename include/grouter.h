@@ -135,6 +135,27 @@ int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const int32_t* fold
                          int32_t E_tgt, int32_t* counts, int32_t* offsets, int32_t* row_to_slot, int32_t* slot_to_row,
                          int32_t* status, void* stream);
 
+/* Router head: writes the pre-dispatch routing cache from router hidden states (the step before grouter_plan; in
+ * the paper it runs once over the corpus, in the data pipeline).  Eq. 2, section "Mixture-of-Experts":
+ *   r(x) = g(TopK(s(x), k)),   s(x) = W~_s^T h,   W~_s = W_s M   (section "Expert Folding", Matrix Folding)
+ * with the fold applied to the scores BEFORE TopK (a token never picks one target twice), unlike the id fold of
+ * grouter_plan.  g is a softmax over the k kept scores or a sigmoid of each.
+ *   H         [T, d_h] bf16 router hidden states          W_s   [E_src, d_h] bf16 score layer, one row per source expert
+ *   fold_map  [E_src] int32 in [0,E_tgt): the j with M_ij = 1, or NULL (E_src == E_tgt)
+ *   idx_out   [T,k] uint8: kept experts, scores descending, equal scores by ascending id
+ *   gates_out [T,k] bf16:  r(x) of the kept experts, round-to-nearest-even
+ *   scores_out [T,E_tgt] f32 folded scores, or NULL       workspace: grouter_route_workspace_bytes(T, E_src, E_tgt) bytes, 256-aligned
+ *   status    device int32 the kernels OR bits into: 1 = a fold target was out of range (counted as target 0),
+ *             2 = a bounded wait in the score GEMM ran out.  The caller zeroes it.
+ * Required: T, d_h, E_src multiples of 8; E_tgt <= 256 (uint8 ids); E_src <= 1024; k <= min(32, E_tgt); finite inputs.
+ * Scores are accumulated in fp32; where two scores differ by less than fp32 rounding the kept set may differ from an
+ * exact evaluation.  Errors: INVALID_ARG, UNSUPPORTED, MISALIGNED, CUDA. */
+enum { GROUTER_NORM_SOFTMAX = 0, GROUTER_NORM_SIGMOID = 1 };
+size_t grouter_route_workspace_bytes(int32_t T, int32_t E_src, int32_t E_tgt);
+int grouter_route(const void* H, const void* W_s, const int32_t* fold_map, int32_t T, int32_t d_h, int32_t E_src, int32_t E_tgt,
+                  int32_t k, int32_t norm, void* idx_out, void* gates_out, float* scores_out, void* workspace, int32_t* status,
+                  void* stream);
+
 /* Forward, Eq. 1:  Y[t,:] = sum_j gates[t,j] * f_{e(t,j)}(X[t,:]).
  *   X     [T,d] bf16             gates [T,k] bf16 or f32 (dims.gate_dtype), used as given
  *   W_gu  [E_tgt, 2*ffn, d] bf16: rows 0..ffn-1 gate projection, ffn..2ffn-1 up projection

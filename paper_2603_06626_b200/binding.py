@@ -16,11 +16,12 @@ from . import build as _build
 
 IDX_U8, IDX_I32 = 0, 1
 FLAG_ACCUMULATE_DW = 1
+NORM_SOFTMAX, NORM_SIGMOID = 0, 1
 GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
-           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait"]
+           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW"]
 
@@ -67,6 +68,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_moe_bwd.restype = ctypes.c_int
     lib.grouter_moe_step_host.argtypes = [vp] * 15
     lib.grouter_moe_step_host.restype = ctypes.c_int
+    lib.grouter_route_workspace_bytes.argtypes = [ctypes.c_int32] * 3
+    lib.grouter_route_workspace_bytes.restype = ctypes.c_size_t
+    lib.grouter_route.argtypes = [vp, vp, i32p] + [ctypes.c_int32] * 6 + [vp, vp, f32p, vp, i32p, vp]
+    lib.grouter_route.restype = ctypes.c_int
     lib.grouter_host_wait.argtypes = [vp, ctypes.c_int32]
     lib.grouter_host_wait.restype = ctypes.c_int
     lib.grouter_status.argtypes = [vp, vp]
@@ -195,6 +200,29 @@ class GrouterLayer:
 
     def check_status(self) -> None:
         _check(self.status(), "device status")
+
+
+def route(H: torch.Tensor, W_s: torch.Tensor, fold_map: Optional[torch.Tensor], E_tgt: int, k: int, norm: int = NORM_SOFTMAX,
+          want_scores: bool = False):
+    """Router head (grouter_route): H [T,d_h] bf16, W_s [E_src,d_h] bf16 -> (idx uint8 [T,k], gates bf16 [T,k],
+    folded scores f32 [T,E_tgt] or None).  Raises on a device-side status."""
+    lib = load_library()
+    T, d_h = H.shape
+    E_src = W_s.shape[0]
+    dev = H.device
+    idx = torch.empty((T, k), dtype=torch.uint8, device=dev)
+    gates = torch.empty((T, k), dtype=torch.bfloat16, device=dev)
+    scores = torch.empty((T, E_tgt), dtype=torch.float32, device=dev) if want_scores else None
+    ws = torch.empty(max(1, lib.grouter_route_workspace_bytes(T, E_src, E_tgt)), dtype=torch.uint8, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib.grouter_route(_ptr(H), _ptr(W_s), _ptr(fold_map), T, d_h, E_src, E_tgt, k, norm, _ptr(idx), _ptr(gates), _ptr(scores),
+                                 _ptr(ws), _ptr(status), _stream()), "grouter_route")
+        torch.cuda.synchronize(dev)
+    st = int(status.item())
+    if st != 0:
+        raise GrouterError(-7 if st & 2 else -6, "grouter_route device status")
+    return idx, gates, scores
 
 
 def plan_noalloc(idx: torch.Tensor, fold_map: Optional[torch.Tensor], E_src: int, E_tgt: int, out=None, status=None):
