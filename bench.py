@@ -130,6 +130,42 @@ def router_head_leg(dev, T=32768, d_h=512, E_src=128, E_tgt=128, k=8, iters=20):
             "gbs": by / (ms * 1e-3) / 1e9, "gpu_launches_per_call": 3}
 
 
+def routing_stats_leg(dev, idx, E, seq_len=4096, n_nodes=8, iters=20):
+    """Loads, co-activation matrix, affinity vectors, MaxVio and Algorithm-1 placement over the step's routing table.
+    Algorithmic bytes: the ids read once, the statistics written."""
+    import torch
+    from paper_2603_06626_b200 import binding
+    lib = binding.load_library()
+    T, k = idx.shape
+    S = T // seq_len
+    i32 = dict(dtype=torch.int32, device=dev)
+    node = (torch.arange(E, device=dev, dtype=torch.int32) % n_nodes).contiguous()
+    loads, coact = torch.empty(E, **i32), torch.empty((E, E), **i32)
+    phi, mv = torch.empty((S, E), dtype=torch.float32, device=dev), torch.empty(1, dtype=torch.float32, device=dev)
+    lt, bn, status = torch.empty((S, n_nodes), **i32), torch.empty(S, **i32), torch.zeros(1, **i32)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        rc = lib.grouter_routing_stats(idx.data_ptr(), binding.IDX_U8, T, k, E, seq_len, node.data_ptr(), n_nodes, loads.data_ptr(),
+                                       coact.data_ptr(), phi.data_ptr(), mv.data_ptr(), lt.data_ptr(), bn.data_ptr(), status.data_ptr(), st)
+        assert rc == 0, rc
+
+    for _ in range(3):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and int(loads.sum().item()) == T * k
+    ms = e0.elapsed_time(e1) / iters
+    by = T * k * 1.0 + 4.0 * (E + E * E + S * E + S * n_nodes + S)
+    return {"T": T, "k": k, "E": E, "seq_len": seq_len, "n_nodes": n_nodes, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
+            "algorithmic_bytes": by, "gbs": by / (ms * 1e-3) / 1e9, "max_vio": float(mv.item())}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -462,6 +498,8 @@ def main():
         rh = router_head_leg(dev)
         rh["frac_of_hbm"] = rh["gbs"] / peaks["hbm_gbs"]
         line["router_head"] = rh
+        if w.E_src <= 256 and w.T % 4096 == 0:
+            line["routing_stats"] = routing_stats_leg(dev, idx, w.E_src)
     if world == 1 and not args.no_cpu_baseline:
         v, dt, threads = oracle_sample_tokens_per_sec(w, li, args.cpu_baseline_tokens)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,

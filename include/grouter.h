@@ -156,6 +156,30 @@ int grouter_route(const void* H, const void* W_s, const int32_t* fold_map, int32
                   int32_t k, int32_t norm, void* idx_out, void* gates_out, float* scores_out, void* workspace, int32_t* status,
                   void* stream);
 
+/* Routing statistics of a cached routing table (inputs of the method's offline stages; see the sections "Expert
+ * Folding", "Decoupling Communication Optimization", the appendices "Maximal Violation" and "Efficiency Experiment
+ * Detail", Algorithm 1).  Samples are consecutive runs of seq_len tokens; S = T / seq_len.  A token's repeated id
+ * counts once.
+ *   idx          [T,k] uint8 or int32 (idx_dtype), values in [0,E)
+ *   node_of_expert [E] int32 in [0,n_nodes), or NULL when local_tokens and best_node are NULL
+ *   loads        [E] int32 out: tokens per expert L_i              max_vio [1] f32 out: (max L - mean L) / mean L
+ *   coact        [E,E] int32 out: P_ij = tokens activating both i and j (diagonal: L_i)
+ *   phi          [S,E] f32 out: routing affinity vectors, phi(X)_i = (1/|X|) #{t in X : expert i kept}
+ *   local_tokens [S,n_nodes] int32 out or NULL: tokens of the sample with at least one kept expert on the node
+ *   best_node    [S] int32 out or NULL: the node with the most local tokens (lowest-numbered among equals)
+ *   status       device int32, bit 1 ORed in when an id or node number is out of range (that entry is skipped); caller zeroes it
+ * Required: T a multiple of seq_len, k <= 32, E <= 1024 (256 for uint8 ids), n_nodes <= 64.  All outputs are device
+ * pointers and are overwritten.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int grouter_routing_stats(const void* idx, int32_t idx_dtype, int32_t T, int32_t k, int32_t E, int32_t seq_len,
+                          const int32_t* node_of_expert, int32_t n_nodes, int32_t* loads, int32_t* coact, float* phi, float* max_vio,
+                          int32_t* local_tokens, int32_t* best_node, int32_t* status, void* stream);
+/* Greedy affinity folding (section "Expert Folding", Expert Folding Mapping), on the HOST: from the co-activation
+ * matrix coact_host [E_src,E_src] to fold_map_host [E_src] -> [0,E_tgt).  Groups hold floor(E_src/E_tgt) experts, the
+ * first E_src mod E_tgt of them one more; a group is opened by the lowest-numbered unassigned expert and grown by the
+ * unassigned expert with the largest summed co-activation with its members (lower id on equal sums); target j is
+ * group j.  Needs E_tgt <= E_src.  Plain host arrays; no GPU work. */
+int grouter_fold_greedy_host(const int32_t* coact_host, int32_t E_src, int32_t E_tgt, int32_t* fold_map_host);
+
 /* Forward, Eq. 1:  Y[t,:] = sum_j gates[t,j] * f_{e(t,j)}(X[t,:]).
  *   X     [T,d] bf16             gates [T,k] bf16 or f32 (dims.gate_dtype), used as given
  *   W_gu  [E_tgt, 2*ffn, d] bf16: rows 0..ffn-1 gate projection, ffn..2ffn-1 up projection

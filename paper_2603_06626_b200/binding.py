@@ -21,7 +21,8 @@ GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
-           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes"]
+           "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
+           "grouter_fold_greedy_host"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW"]
 
@@ -72,6 +73,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_route_workspace_bytes.restype = ctypes.c_size_t
     lib.grouter_route.argtypes = [vp, vp, i32p] + [ctypes.c_int32] * 6 + [vp, vp, f32p, vp, i32p, vp]
     lib.grouter_route.restype = ctypes.c_int
+    lib.grouter_routing_stats.argtypes = [vp] + [ctypes.c_int32] * 5 + [i32p, ctypes.c_int32, i32p, i32p, f32p, f32p, i32p, i32p, i32p, vp]
+    lib.grouter_routing_stats.restype = ctypes.c_int
+    lib.grouter_fold_greedy_host.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp]
+    lib.grouter_fold_greedy_host.restype = ctypes.c_int
     lib.grouter_host_wait.argtypes = [vp, ctypes.c_int32]
     lib.grouter_host_wait.restype = ctypes.c_int
     lib.grouter_status.argtypes = [vp, vp]
@@ -223,6 +228,39 @@ def route(H: torch.Tensor, W_s: torch.Tensor, fold_map: Optional[torch.Tensor], 
     if st != 0:
         raise GrouterError(-7 if st & 2 else -6, "grouter_route device status")
     return idx, gates, scores
+
+
+def routing_stats(idx: torch.Tensor, E: int, seq_len: int, node_of_expert: Optional[torch.Tensor] = None, n_nodes: int = 0):
+    """grouter_routing_stats: -> dict(loads, coact, phi, max_vio[, local_tokens, best_node]) of device tensors."""
+    lib = load_library()
+    T, k = idx.shape
+    dev = idx.device
+    S = T // max(seq_len, 1)
+    i32 = dict(dtype=torch.int32, device=dev)
+    out = dict(loads=torch.empty(E, **i32), coact=torch.empty((E, E), **i32), phi=torch.empty((S, E), dtype=torch.float32, device=dev),
+               max_vio=torch.empty(1, dtype=torch.float32, device=dev))
+    if node_of_expert is not None:
+        out["local_tokens"] = torch.empty((S, n_nodes), **i32)
+        out["best_node"] = torch.empty(S, **i32)
+    status = torch.zeros(1, **i32)
+    with torch.cuda.device(dev):
+        _check(lib.grouter_routing_stats(_ptr(idx), IDX_U8 if idx.dtype == torch.uint8 else IDX_I32, T, k, E, seq_len, _ptr(node_of_expert),
+                                         n_nodes, _ptr(out["loads"]), _ptr(out["coact"]), _ptr(out["phi"]), _ptr(out["max_vio"]),
+                                         _ptr(out.get("local_tokens")), _ptr(out.get("best_node")), _ptr(status), _stream()),
+               "grouter_routing_stats")
+        torch.cuda.synchronize(dev)
+    out["status"] = int(status.item())
+    return out
+
+
+def fold_greedy(coact, E_tgt: int):
+    """grouter_fold_greedy_host: host int32 co-activation matrix [E_src,E_src] (numpy) -> fold_map int32 [E_src] (numpy)."""
+    import numpy as np
+    lib = load_library()
+    P = np.ascontiguousarray(coact, dtype=np.int32)
+    fold = np.empty(P.shape[0], dtype=np.int32)
+    _check(lib.grouter_fold_greedy_host(P.ctypes.data, P.shape[0], E_tgt, fold.ctypes.data), "grouter_fold_greedy_host")
+    return fold
 
 
 def plan_noalloc(idx: torch.Tensor, fold_map: Optional[torch.Tensor], E_src: int, E_tgt: int, out=None, status=None):
