@@ -166,7 +166,7 @@ int grouter_route(const void* H, const void* W_s, const int32_t* fold_map, int32
  *   coact        [E,E] int32 out: P_ij = tokens activating both i and j (diagonal: L_i)
  *   phi          [S,E] f32 out: routing affinity vectors, phi(X)_i = (1/|X|) #{t in X : expert i kept}
  *   local_tokens [S,n_nodes] int32 out or NULL: tokens of the sample with at least one kept expert on the node
- *   best_node    [S] int32 out or NULL: the node with the most local tokens (lowest-numbered among equals)
+ *   best_node    [S] int32 out or NULL: the node with the most local tokens (lowest-numbered among equals); needs local_tokens
  *   status       device int32, bit 1 ORed in when an id or node number is out of range (that entry is skipped); caller zeroes it
  * Required: T a multiple of seq_len, k <= 32, E <= 1024 (256 for uint8 ids), n_nodes <= 64.  All outputs are device
  * pointers and are overwritten.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */

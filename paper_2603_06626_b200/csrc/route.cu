@@ -67,9 +67,13 @@ __global__ void __launch_bounds__(ROUTE_THREADS) route_topk_kernel(const float* 
       const int j = lane + 32 * q;
       float acc = -INFINITY;
       if (j < E_tgt) {
-        acc = 0.f;
-        const int b = __ldg(grp_off + j), e = __ldg(grp_off + j + 1);
-        for (int p = b; p < e; ++p) acc += mine[__ldg(grp_src + p)];
+        if (grp_off == nullptr) {       // no fold: target j is source j
+          acc = mine[j];
+        } else {
+          acc = 0.f;
+          const int b = __ldg(grp_off + j), e = __ldg(grp_off + j + 1);
+          for (int p = b; p < e; ++p) acc += mine[__ldg(grp_src + p)];
+        }
         if (scores_out) scores_out[(size_t)t * E_tgt + j] = acc;
       }
       v[q] = acc;
@@ -179,8 +183,12 @@ int grouter_route(const void* H, const void* W_s, const int32_t* fold_map, int32
   int32_t* grp_src = reinterpret_cast<int32_t*>(base + w.grp_src);
   // source scores: [T, d_h] x [E_src, d_h]^T on the tensor cores, fp32 out
   if (launch_dense_gemm(H, 0, W_s, 0, S_src, T, E_src, d_h, status, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  route_groups_kernel<<<1, ROUTE_THREADS, 0, st>>>(fold_map, E_src, E_tgt, grp_off, grp_src, status);
-  if (cudaGetLastError() != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (fold_map) {
+    route_groups_kernel<<<1, ROUTE_THREADS, 0, st>>>(fold_map, E_src, E_tgt, grp_off, grp_src, status);
+    if (cudaGetLastError() != cudaSuccess) return GROUTER_ERR_CUDA;
+  } else {
+    grp_off = nullptr;
+  }
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
