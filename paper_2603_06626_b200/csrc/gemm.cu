@@ -16,7 +16,11 @@
 // complete on the leader CTA's barrier); warp 1 of the leader CTA issues the MMAs for the pair into one of two
 // 256-column TMEM accumulators (present in both CTAs) and releases stages / publishes accumulators to both
 // CTAs with multicast commits; warps 2-9 of each CTA drain the other accumulator with tcgen05.ld and run the
-// fused epilogue on their CTA's 128 rows, so the epilogue of tile i overlaps the main loop of tile i+1.
+// fused epilogue on their CTA's 128 rows, so the epilogue of tile i overlaps the main loop of tile i+1.  bf16 outputs
+// leave through swizzled shared-memory staging blocks and TMA tile stores; fp32 outputs (weight gradients) are read
+// from TMEM in the MMA-fragment arrangement, where four neighbouring threads own a 32-byte run of a row, and go
+// straight to global memory in full sectors: the main loop runs at the shared-memory bandwidth, so every staged
+// byte the epilogue avoids is main-loop time won.
 // Operands may be K-major (rows of the stored matrix run along K) or MN-major (rows run along M/N); both are
 // described to the MMA by shared-memory descriptors, so no operand is ever transposed in memory.
 //
@@ -62,7 +66,7 @@ struct GemmParams {
   int32_t gate_is_f32;
   const __nv_bfloat16* in_G;   // DH
   const __nv_bfloat16* in_U;   // DH
-  float* out_f;                // DH: dgate_part
+  float* out_f;                // DH: dgate_part; weight gradients / DENSE: the fp32 output [E, M, N]
   int32_t* status;
 };
 
@@ -377,15 +381,6 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ptx::bulk_commit();
       }
     };
-    auto stage_send_3d = [&](uint32_t blk, const CUtensorMap* tm, int x, int y, int z, bool add) {
-      ptx::fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-        if (add) ptx::tma_reduce_add_3d(tm, blk, x, y, z);
-        else ptx::tma_store_3d(tm, blk, x, y, z, stream_out);
-        ptx::bulk_commit();
-      }
-    };
     // DH: saved pre-activations G and U of one 32-column chunk of this thread's row (zeros beyond F)
     auto load_gu = [&](const Tile& ti, int c, uint4 (&g4)[4], uint4 (&u4)[4]) {
       const int c0 = half * 128 + c * 32;
@@ -526,27 +521,40 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const int nt = ti.col0 / BN;
           p.out_f[(size_t)(nt * 2 + half) * p.R_pad_max + (size_t)ti.row0 + r] = dgate;
         }
-      } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile, four 32-column blocks per warp
-        // (an expert without rows has nothing to add when accumulating; otherwise its tile is stored as zeros)
-        if (y0 < ti.row0 + ti.m_valid && (have_acc || !ti.add)) {
+      } else {  // WGRAD_D, WGRAD_GU, DENSE: fp32 tile straight from TMEM to global memory (stored, or added for a partial sum)
+        if (ti.m_valid > quad * 32 && (have_acc || !ti.add)) {
 #pragma unroll
-          for (int blk = 0; blk < 4; ++blk) {
-            const int cb = half * 128 + blk * 32;
-            if (ti.n_valid - cb > 0) {
-              const uint32_t sb = flip ? blk_b : blk_a;   // not the block of the previous store
-              flip ^= 1u;
-              uint32_t ra[32];
-              if (have_acc) {
-                ptx::tmem_ld32(t_row + cb, ra);
-                ptx::tmem_ld_wait();
-              } else {
+          for (int rh = 0; rh < 2; ++rh) {
+            const int ra_row = quad * 32 + rh * 16 + (lane >> 2), rb_row = ra_row + 8;
+            float* pa = p.out_f + ((size_t)ti.e * p.M + (size_t)(ti.row0 + ra_row)) * p.N + ti.col0;
+            float* pb = pa + (size_t)8 * p.N;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) ra[i] = 0u;
+            for (int cc = 0; cc < 4; ++cc) {
+              const int c0 = half * 128 + cc * 32;
+              if (ti.n_valid - c0 > 0) {
+                uint32_t r[16];
+                if (have_acc) {
+                  ptx::tmem_ld_16x256b_x4(tmem_base + (uint32_t)acc * BN + ((uint32_t)(quad * 32 + rh * 16) << 16) + c0, r);
+                  ptx::tmem_ld_wait();
+                } else {
+#pragma unroll
+                  for (int i = 0; i < 16; ++i) r[i] = 0u;
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const int col = c0 + 8 * j + 2 * (lane & 3);
+                  if (col < ti.n_valid) {
+                    if (ra_row < ti.m_valid) {
+                      if (ti.add) ptx::red_add_v2_f32(pa + col, r[4 * j], r[4 * j + 1]);
+                      else ptx::st_global_v2_stream(pa + col, r[4 * j], r[4 * j + 1]);
+                    }
+                    if (rb_row < ti.m_valid) {
+                      if (ti.add) ptx::red_add_v2_f32(pb + col, r[4 * j + 2], r[4 * j + 3]);
+                      else ptx::st_global_v2_stream(pb + col, r[4 * j + 2], r[4 * j + 3]);
+                    }
+                  }
+                }
               }
-              stage_wait_older();
-#pragma unroll
-              for (int q = 0; q < 8; ++q) stage_put(sb, q, ra[q * 4], ra[q * 4 + 1], ra[q * 4 + 2], ra[q * 4 + 3]);
-              stage_send_3d(sb, &tmC0, ti.col0 + cb, y0, ti.e, ti.add);
             }
           }
         }
@@ -612,19 +620,6 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t 
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
-}
-
-// fp32 tensor [batch, rows, cols]; box = {32 columns, 32 rows, 1}: the epilogue's store block.
-static bool make_map_f32_out(CUtensorMap* tm, const void* base, uint64_t batch, uint64_t rows, uint64_t cols) {
-  EncodeTiledFn fn = get_encode_fn();
-  if (!fn) return false;
-  cuuint64_t gdim[3] = {cols, rows, batch};
-  cuuint64_t gstr[2] = {cols * 4, rows * cols * 4};
-  cuuint32_t box[3] = {32, 32, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -702,17 +697,16 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
       if (!ok) return cudaErrorInvalidValue;
       return launch_t<MODE_DX, false, true>(m, p, grid, st);
     case MODE_WGRAD_D:
-      ok = make_map(&m.A, ws.dYp, Rp, d, 64) && make_map(&m.B, ws.Hs, Rp, F, 64) && make_map_f32_out(&m.C0, dW_d, E, d, F);
-      m.C1 = m.C2 = m.C0;
-      p.M = d; p.N = F;
+      ok = make_map(&m.A, ws.dYp, Rp, d, 64) && make_map(&m.B, ws.Hs, Rp, F, 64);
+      m.C0 = m.C1 = m.C2 = m.A;   // fp32 tiles are stored without a tensor map
+      p.M = d; p.N = F; p.out_f = dW_d;
       p.tiles_m = cdiv(d, PM); p.tiles_n = cdiv(F, BN);
       if (!ok) return cudaErrorInvalidValue;
       return launch_t<MODE_WGRAD_D, true, true>(m, p, grid, st);
     case MODE_WGRAD_GU:
-      ok = make_map(&m.A, ws.dGU, Rp, 2 * (uint64_t)F, 64) && make_map(&m.B, ws.Xp, Rp, d, 64) &&
-           make_map_f32_out(&m.C0, dW_gu, E, 2 * (uint64_t)F, d);
-      m.C1 = m.C2 = m.C0;
-      p.M = 2 * F; p.N = d;
+      ok = make_map(&m.A, ws.dGU, Rp, 2 * (uint64_t)F, 64) && make_map(&m.B, ws.Xp, Rp, d, 64);
+      m.C0 = m.C1 = m.C2 = m.A;
+      p.M = 2 * F; p.N = d; p.out_f = dW_gu;
       p.tiles_m = cdiv(2 * F, PM); p.tiles_n = cdiv(d, BN);
       if (!ok) return cudaErrorInvalidValue;
       return launch_t<MODE_WGRAD_GU, true, true>(m, p, grid, st);
@@ -755,11 +749,12 @@ cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, 
   p.tiles_m = cdiv(M, PM);
   p.tiles_n = cdiv(N, BN);
   p.status = status;
+  p.out_f = C;
   Maps m;
   const bool ok = (a_mn ? make_map(&m.A, A, K, M, 64) : make_map(&m.A, A, M, K, 128)) &&
-                  (b_mn ? make_map(&m.B, B, K, N, 64) : make_map(&m.B, B, N, K, 128)) && make_map_f32_out(&m.C0, C, 1, M, N);
+                  (b_mn ? make_map(&m.B, B, K, N, 64) : make_map(&m.B, B, N, K, 128));
   if (!ok) return cudaErrorInvalidValue;
-  m.C1 = m.C2 = m.C0;
+  m.C0 = m.C1 = m.C2 = m.A;
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);

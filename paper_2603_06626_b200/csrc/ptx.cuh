@@ -129,21 +129,6 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t sme
                "r"(smem_src), "r"(x), "r"(y), "l"(l2_policy)
                : "memory");
 }
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t smem_src, int32_t x, int32_t y, int32_t z,
-                                             uint64_t l2_policy) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;" ::"l"(
-                   reinterpret_cast<uint64_t>(tm)),
-               "r"(smem_src), "r"(x), "r"(y), "r"(z), "l"(l2_policy)
-               : "memory");
-}
-// Tile reduction shared -> global: every element of the tile is added to the element in global memory (the
-// element type, f32 here, comes from the tensor map); out-of-bounds parts are clipped like a store.
-__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* tm, uint32_t smem_src, int32_t x, int32_t y, int32_t z) {
-  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(
-                   reinterpret_cast<uint64_t>(tm)),
-               "r"(smem_src), "r"(x), "r"(y), "r"(z)
-               : "memory");
-}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // the shared-memory sources of all committed groups have been read
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
@@ -205,6 +190,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
+}
+// 16 lanes x 32 columns in the MMA-fragment arrangement: for j = 0..3, thread t holds columns 8j + 2(t%4), +1 of lane
+// t/4 in r[4j], r[4j+1] and of lane t/4 + 8 in r[4j+2], r[4j+3]: four neighbouring threads own one 32-byte run of a row.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void st_global_v2_stream(float* p, uint32_t a, uint32_t b) {
+  asm volatile("st.global.cs.v2.b32 [%0], {%1, %2};" ::"l"(p), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ void red_add_v2_f32(float* p, uint32_t a, uint32_t b) {
+  asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
