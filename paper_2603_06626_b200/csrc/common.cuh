@@ -51,7 +51,7 @@ struct PaddedPlan {
   int32_t* pair_expert;   // [max_m_tiles] expert of the tile; bit 30 set when the second half holds rows of that expert
   int32_t* n_pair_tiles;  // [1]
   // Work list of the weight-gradient GEMMs: one entry per (expert, chunk of rows).  An expert with several
-  // chunks accumulates them into its pre-zeroed gradient with reduce-add stores; a one-chunk expert stores.
+  // chunks adds them into its pre-zeroed gradient (vector reductions to global memory); a one-chunk expert stores.
   int32_t* wchunk_expert; // [max_wchunks] expert | WCHUNK_SPLIT
   int32_t* wchunk_row0;   // [max_wchunks] first padded row of the chunk
   int32_t* wchunk_rows;   // [max_wchunks] rows in the chunk (multiple of 128; 0 for an expert without slots)
