@@ -42,13 +42,16 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 def kernel_source_tag() -> str:
-    """Short hash of the CUDA sources: DRAM counters taken with another build are not reported."""
+    """Short hash of the CUDA sources (comments and blank space left out): DRAM counters taken with other code are not
+    reported."""
     import hashlib
+    import re
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2603_06626_b200", "csrc")
     for name in sorted(os.listdir(csrc)):
-        with open(os.path.join(csrc, name), "rb") as f:
-            h.update(name.encode() + b"\0" + f.read())
+        with open(os.path.join(csrc, name)) as f:
+            code = re.sub(r"//[^\n]*", "", f.read())
+        h.update(name.encode() + b"\0" + "".join(code.split()).encode())
     return h.hexdigest()[:12]
 
 
