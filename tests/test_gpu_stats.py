@@ -55,11 +55,13 @@ def test_greedy_fold_on_host_matches_oracle_and_feeds_the_router():
     w = synth.WORKLOADS["fine_fold"]
     idx = synth.make_idx(w)[:4096]
     P = binding.routing_stats(to_dev(idx), w.E_src, 1024)["coact"].cpu().numpy()
+    P_oracle = so.coactivation(idx, w.E_src)              # the oracle folds its own matrix, never the CUDA path's
+    assert np.array_equal(P, P_oracle)
     for E_T in (16, 24, 64, 1):
         fold = binding.fold_greedy(P, E_T)
-        assert np.array_equal(fold, so.greedy_fold(P, E_T))
+        assert np.array_equal(fold, so.greedy_fold(P_oracle, E_T))
     rng = np.random.default_rng(1)
     A = rng.integers(0, 1000, size=(37, 37))
     assert np.array_equal(binding.fold_greedy(A + A.T, 5), so.greedy_fold(A + A.T, 5))
     with pytest.raises(binding.GrouterError):
-        binding.fold_greedy(P, w.E_src + 1)
+        binding.fold_greedy(P_oracle, w.E_src + 1)
