@@ -54,7 +54,7 @@ struct PaddedPlan {
   // chunks adds them into its pre-zeroed gradient (vector reductions to global memory); a one-chunk expert stores.
   int32_t* wchunk_expert; // [max_wchunks] expert | WCHUNK_SPLIT
   int32_t* wchunk_row0;   // [max_wchunks] first padded row of the chunk
-  int32_t* wchunk_rows;   // [max_wchunks] rows in the chunk (multiple of 128; 0 for an expert without slots)
+  int32_t* wchunk_rows;   // [max_wchunks] rows in the chunk (multiple of 64; 0 for an expert without slots)
   int32_t* n_wchunks;     // [1]
   int32_t* slot_to_prow;  // [R]
   int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows

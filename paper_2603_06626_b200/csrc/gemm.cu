@@ -54,7 +54,7 @@ struct GemmParams {
   const int32_t* n_wchunks;    // device scalar: (expert, row chunk) entries (weight-gradient modes)
   const int32_t* wchunk_expert;// device [chunks] expert | WCHUNK_SPLIT
   const int32_t* wchunk_row0;  // device [chunks] first padded row
-  const int32_t* wchunk_rows;  // device [chunks] rows, multiple of 128
+  const int32_t* wchunk_rows;  // device [chunks] rows, multiple of 64
   int32_t E, d, F;
   int32_t accumulate;          // weight-gradient modes: add every tile into the caller's gradient
   int32_t M, N, K;             // DENSE: problem; WGRAD: per-expert output M x N

@@ -227,7 +227,12 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
       const int i = s_wch[e] + c;
       pp.wchunk_expert[i] = e | (n > 1 ? WCHUNK_SPLIT : 0);
       pp.wchunk_row0[i] = s_pad[e] + (c * base + min(c, rem)) * ROW_TILE;
-      pp.wchunk_rows[i] = (base + (c < rem ? 1 : 0)) * ROW_TILE;
+      int rows = (base + (c < rem ? 1 : 0)) * ROW_TILE;
+      // the contraction runs in steps of 64 rows: when the expert's last block holds at most 64 real rows, its second
+      // half is all padding (zeros) and is left out
+      const int tail = s_cnt[e] & (ROW_TILE - 1);
+      if (c == n - 1 && tail >= 1 && tail <= ROW_TILE / 2) rows -= ROW_TILE / 2;
+      pp.wchunk_rows[i] = rows;
     }
   }
   // pad rows carry no slot
