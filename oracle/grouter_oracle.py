@@ -18,7 +18,7 @@ What it follows
   * Expert folding (section "Expert Folding", Matrix Folding): the binary
     map M in its compact form fold_map[source id] -> target id.
 
-Readings where the paper is silent (all listed in the design notes):
+Readings where the paper is silent:
   * f_i is a bias-free SwiGLU FFN:  f(x) = W_d ( silu(W_g x) * (W_u x) ),
     silu(z) = z / (1 + exp(-z)).
   * gates are used as given: never renormalised, leaf inputs, so

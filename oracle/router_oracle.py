@@ -13,7 +13,7 @@ What it follows
   * Pre-dispatch cache (appendix "Efficiency Experiment Detail"): per token, k expert ids as uint8 and k routing
     scores as bfloat16.
 
-Readings where the paper is silent (listed in the design notes):
+Readings where the paper is silent:
   * s(x) = W_s^T h with h the router's last hidden state of the token; no bias.
   * TopK order: scores descending, equal scores by ascending expert id; the cache keeps that order.
   * softmax runs over the k kept scores only (the usual "softmax after top-k"); sigmoid is applied to each kept score.

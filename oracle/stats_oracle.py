@@ -14,7 +14,7 @@ What it follows
   * Sample placement, Algorithm 1 (appendix "Efficiency Experiment Detail"): per sample and node, the number of the
     sample's tokens with at least one kept expert on the node; the sample goes to the node where that number is largest.
 
-Readings where the paper is silent or loose (listed in the design notes):
+Readings where the paper is silent or loose:
   * P is the sum over tokens of a a^T with a the token's 0/1 activation vector: off-diagonal entries are pair counts,
     the diagonal holds each expert's activation count (never used by the folding rule, which only looks at other experts).
   * A token that lists one id twice activates that expert once (ids are distinct in the cache the router head writes).
