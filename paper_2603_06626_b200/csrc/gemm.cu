@@ -629,12 +629,15 @@ struct Maps {
 
 template <int MODE, bool A_MN, bool B_MN>
 static cudaError_t launch_t(const Maps& m, const GemmParams& p, int grid, cudaStream_t st) {
-  static bool configured = false;
+  // the opt-in to more than 48 KB of dynamic shared memory is a per-device setting: once per device and instantiation
+  static bool configured[64] = {};
   auto kern = grouped_gemm_kernel<MODE, A_MN, B_MN>;
-  if (!configured) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
     if (e != cudaSuccess) return e;
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   kern<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(m.A, m.B, m.C0, m.C1, m.C2, p);
   return cudaGetLastError();
