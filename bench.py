@@ -330,6 +330,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-plan-scale", action="store_true")
+    ap.add_argument("--no-isolated", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=10)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -405,6 +406,18 @@ def main():
     ms_step = ms_total / args.steps
     value = shard.job_tokens_per_sec(world, w.T, ms_step)
 
+    # ---- every kernel alone: 30 ms of idle time after each launch, so that none starts at the power cap ----
+    isolated = None
+    if world == 1 and not args.no_isolated:
+        layer.timing_gap(30000)
+        layer.timing_enable(len(binding.KERNEL_SLOTS) * 3)
+        for _ in range(3):
+            step()
+        isolated = layer.timing_read()
+        layer.timing_enable(0)
+        layer.timing_gap(0)
+        layer.check_status()
+
     # ---- end to end: host buffers in, host results out, every step ----
     e2e = None
     if not args.no_e2e:
@@ -469,6 +482,15 @@ def main():
         else:
             ent["gbs"] = amount / avg_s / 1e9
             ent["frac_of_hbm"] = ent["gbs"] / peaks["hbm_gbs"]
+        if isolated is not None and isolated.get(name, (0.0, 0))[1] > 0:
+            iso_s = isolated[name][0] / isolated[name][1] * 1e-3
+            ent["alone_ms"] = iso_s * 1e3
+            if kind == "flop":
+                ent["alone_tflops"] = amount / iso_s / 1e12
+                ent["alone_frac_of_burst"] = ent["alone_tflops"] / peaks["bf16_tflops"]
+            else:
+                ent["alone_gbs"] = amount / iso_s / 1e9
+                ent["alone_frac_of_hbm"] = ent["alone_gbs"] / peaks["hbm_gbs"]
         kernels[name] = ent
     dom = max(GEMM_SLOTS, key=lambda k: per_kernel[k][0])
     traffic = recorded_traffic(w.name, dom)
@@ -478,6 +500,9 @@ def main():
                 "unit": "TFLOP/s", "frac": kernels[dom]["tflops"] / peaks["bf16_tflops_sustained"], "traffic": traffic,
                 "peak_source": f"{peak_src} cuBLAS bf16, sustained (kernel timed inside a long step); burst peak "
                                f"{peaks['bf16_tflops']} gives frac {kernels[dom]['tflops'] / peaks['bf16_tflops']:.3f}"}
+    if "alone_tflops" in kernels[dom]:
+        roofline["alone"] = {"achieved": kernels[dom]["alone_tflops"], "peak": peaks["bf16_tflops"], "frac": kernels[dom]["alone_frac_of_burst"],
+                             "note": "the same kernel timed alone (30 ms idle after every launch) against the burst peak"}
     gemm_ms = sum(per_kernel[k][0] for k in GEMM_SLOTS)
     gemm_flops = sum(work[k][1] * per_kernel[k][1] for k in GEMM_SLOTS)
     summary = {"all_gemms_tflops": gemm_flops / (gemm_ms * 1e-3) / 1e12,

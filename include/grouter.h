@@ -239,6 +239,10 @@ const char* grouter_strerror(int code);
  * 11 reduce_dX, 12 zero_split_dW.   total_ms, launches: HOST arrays of GROUTER_NUM_KERNELS entries. */
 #define GROUTER_NUM_KERNELS 13
 int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records);
+/* While timing is enabled, let `microseconds` (0..1000000; 0 = off, the default) of idle time pass on the stream after
+ * every timed kernel, so that each kernel is measured on a GPU that is not already at its power cap: the figure to
+ * hold against a burst peak, where the back-to-back figure belongs with a sustained peak. */
+int grouter_timing_gap(grouter_ctx* ctx, int32_t microseconds);
 int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t* launches);
 
 /* Component check of the tensor-core core used by every grouped GEMM (no

@@ -66,7 +66,10 @@ struct Timed {
     }
   }
   ~Timed() {
-    if (i >= 0) cudaEventRecord(c->ev_stop[i], st);
+    if (i >= 0) {
+      cudaEventRecord(c->ev_stop[i], st);
+      if (c->idle_gap_us > 0) launch_idle(c->idle_gap_us, st);   // the next kernel starts on a GPU that has rested
+    }
   }
 };
 
@@ -162,6 +165,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->ev_slot = nullptr;
   c->ev_cap = c->ev_used = 0;
   c->host_steps = 0;
+  c->idle_gap_us = 0;
   c->s_in = c->s_out = nullptr;
   for (int i = 0; i < 2; ++i) c->ev_in_fwd[i] = c->ev_in_bwd[i] = c->ev_fwd_done[i] = c->ev_bwd_done[i] = c->ev_out_done[i] = nullptr;
   {
@@ -408,6 +412,12 @@ int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records) {
   }
   ctx->ev_cap = n_records;
   ctx->ev_used = 0;
+  return GROUTER_OK;
+}
+
+int grouter_timing_gap(grouter_ctx* ctx, int32_t microseconds) {
+  if (!ctx || microseconds < 0 || microseconds > 1000000) return GROUTER_ERR_INVALID_ARG;
+  ctx->idle_gap_us = microseconds;
   return GROUTER_OK;
 }
 

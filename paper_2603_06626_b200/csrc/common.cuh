@@ -88,6 +88,7 @@ struct grouter_ctx {
   int* ev_slot;
   int ev_cap;
   int ev_used;
+  int idle_gap_us;        // measurement aid: idle time inserted after every timed kernel (0 = none)
 };
 
 namespace grouter {
@@ -123,6 +124,8 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
                                 const void* W_d, float* dW_gu, float* dW_d, cudaStream_t st);
 // Zero-fills dW_gu[e] and dW_d[e] of every expert whose rows are split over several chunks.
 cudaError_t launch_zero_split_dw(grouter_ctx* ctx, float* dW_gu, float* dW_d, cudaStream_t st);
+// A kernel that only lets `microseconds` pass (one thread watching the global timer, capped at one second).
+cudaError_t launch_idle(int microseconds, cudaStream_t st);
 cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,
                               cudaStream_t st);
 

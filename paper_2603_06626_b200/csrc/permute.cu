@@ -133,6 +133,21 @@ __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bf
   }
 }
 
+__global__ void idle_kernel(unsigned long long nanoseconds) {
+  unsigned long long t0, t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  do {
+    __nanosleep(2000);
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  } while (t - t0 < nanoseconds);
+}
+
+cudaError_t launch_idle(int microseconds, cudaStream_t st) {
+  if (microseconds > 1000000) microseconds = 1000000;
+  idle_kernel<<<1, 1, 0, st>>>((unsigned long long)microseconds * 1000ull);
+  return cudaGetLastError();
+}
+
 static int mover_grid(const grouter_ctx* ctx, int T) {
   const int want = (T + MOVE_WARPS - 1) / MOVE_WARPS;
   const int cap = ctx->num_sms * 8;

@@ -104,3 +104,31 @@ def test_host_side_errors():
         layer.forward(X, g, W_gu, W_d)                 # no plan yet
     assert e.value.code == -4
     layer.close()
+
+
+def test_kernel_timing_records_and_idle_gap():
+    """The per-kernel timing aid: one event pair per launch, with or without idle time between launches."""
+    import time
+    from paper_2603_06626_b200 import binding
+    w = synth.WORKLOADS["tiny"]
+    idx = to_dev(synth.make_idx(w))
+    layer = binding.GrouterLayer(w.T, 64, 64, w.E_src, w.k)
+    layer.plan(idx)
+    layer.timing_enable(8)
+    layer.timing_gap(20000)                    # 20 ms after each of the two plan kernels
+    torch.cuda.synchronize()
+    t0 = time.time()
+    layer.plan(idx)
+    rec = layer.timing_read()
+    waited = time.time() - t0
+    assert rec["plan_hist"][1] == 1 and rec["plan_permute"][1] == 1 and rec["plan_hist"][0] > 0
+    assert rec["plan_hist"][0] < 5.0           # the idle time is not part of the kernel's own record
+    assert waited >= 0.035
+    layer.timing_gap(0)
+    layer.plan(idx)
+    assert layer.timing_read()["plan_permute"][1] == 1
+    layer.timing_enable(0)
+    with pytest.raises(binding.GrouterError):
+        layer.timing_gap(-1)
+    assert layer.status() == 0
+    layer.close()
