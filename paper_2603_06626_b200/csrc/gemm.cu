@@ -129,11 +129,20 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
     }
   } else if (MODE == MODE_WGRAD_D || MODE == MODE_WGRAD_GU) {
     // all output tiles of one (expert, row chunk) are adjacent in the schedule: the CTA pairs in flight read the
-    // same chunk of operand rows, which therefore stays in L2 however long the expert's row list is
+    // same chunk of operand rows, which therefore stays in L2 however long the expert's row list is.  A chunk's
+    // tiles take more than one round of the CTA pairs; the operand whose slabs the inner loop walks is fetched
+    // again in every round, so the inner loop runs along the dimension with fewer tiles.
     const int per = p.tiles_m * p.tiles_n;
     const int ci = t / per;
     const int r = t - ci * per;
-    const int mt = r / p.tiles_n, nt = r - mt * p.tiles_n;
+    int mt, nt;
+    if (p.tiles_m < p.tiles_n) {
+      nt = r / p.tiles_m;
+      mt = r - nt * p.tiles_m;
+    } else {
+      mt = r / p.tiles_n;
+      nt = r - mt * p.tiles_n;
+    }
     const int we = __ldg(p.wchunk_expert + ci);
     ti.e = we & ~WCHUNK_SPLIT;
     ti.add = (we & WCHUNK_SPLIT) != 0 || p.accumulate != 0;
