@@ -213,6 +213,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.prow_to_slot = reinterpret_cast<int32_t*>(b + o_p2s);
   c->pp.blk_prefix = reinterpret_cast<int32_t*>(b + o_bp);
   c->pp.ticket = reinterpret_cast<unsigned int*>(b + o_tk);
+  c->pp.tile_counter = c->pp.ticket + 4;   // same 256-byte slot
   c->pp.status = reinterpret_cast<int32_t*>(b + o_st);
   *out = c;
   return GROUTER_OK;

@@ -60,6 +60,7 @@ struct PaddedPlan {
   int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows
   int32_t* blk_prefix;    // [E_tgt * nblk] per-block histogram, then exclusive prefix over blocks
   unsigned int* ticket;   // [1] last-block-done counter
+  unsigned int* tile_counter;   // [1] next tile of the running grouped GEMM; zero between launches
   int32_t* status;        // [1] sticky status bits
 };
 

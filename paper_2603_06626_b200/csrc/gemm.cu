@@ -43,7 +43,7 @@ constexpr int ATOM_BYTES = 64 * BK * 2;         // one 64x64 bf16 box = 8 KB
 constexpr int EPI_WARPS = 8;                    // two warps per TMEM lane quadrant, each takes half of the columns
 constexpr int GEMM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int EPI_STAGE_BYTES = 32 * 128;       // one staging block: 32 rows x 128 bytes; two per epilogue warp
-constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + EPI_WARPS * 2 * EPI_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int GEMM_SMEM = STAGES * STAGE_BYTES + EPI_WARPS * 2 * EPI_STAGE_BYTES + 1024 /*align*/ + 256 /*barriers, tile queue*/;
 constexpr uint32_t TMEM_COLS = 512;
 
 struct GemmParams {
@@ -68,6 +68,7 @@ struct GemmParams {
   const __nv_bfloat16* in_U;   // DH
   float* out_f;                // DH: dgate_part; weight gradients / DENSE: the fp32 output [E, M, N]
   int32_t* status;
+  unsigned int* tile_counter;  // device scalar, zero at launch (unused by DENSE, which has no context to keep one)
 };
 
 struct Tile {     // one CTA's share of a pair tile
@@ -213,6 +214,19 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+  // Tile queue (all modes but DENSE).  The pair takes its tiles from a grid-wide counter instead of a fixed stride: the
+  // pairs then always work on neighbouring tiles of the list, whatever their individual pace, so the operand rows the
+  // neighbours share are fetched from DRAM once.  The leader's producer draws the numbers (two tiles ahead, so the
+  // round trip of the atomic is never waited for) and writes them into a ring of TQ 8-byte slots {sequence, tile} in
+  // both CTAs; the other roles poll their CTA's copy: slot i % TQ holds the pair's i-th tile once its sequence word
+  // reads i + 1.  Nobody acknowledges a slot, because nobody can fall TQ tiles behind: every tile passes at least one
+  // stage through the operand ring (the producer is at most STAGES tiles ahead of the issuer), and the issuer starts a
+  // tile only after every epilogue warp has finished the tile two before it, so the oldest number still unread is at
+  // most STAGES + 3 tiles older than the newest one written (STAGES + 4 <= TQ slots in use).
+  constexpr bool DYN = MODE != MODE_DENSE;
+  constexpr int TQ = 16;
+  static_assert(STAGES + 4 <= TQ && (TQ & (TQ - 1)) == 0, "tile queue too short for the operand ring");
+  auto tq_slot = [&](int i) { return bar_base + 8u * (2 * STAGES + 4) + 8u * (uint32_t)(i & (TQ - 1)); };
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort;
 
@@ -232,6 +246,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       ptx::mbar_init(tfull_bar(a), 1);
       ptx::mbar_init(tempty_bar(a), 2 * EPI_WARPS);
     }
+    for (int q = 0; q < TQ; ++q) ptx::st_shared_volatile_v2(tq_slot(q), 0u, 0u);   // sequence 0: nothing published
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
@@ -254,39 +269,108 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // L2 residency: B (an expert's weights, or the row chunk every output tile of a weight gradient reads) is
   // reused by other CTA pairs and later tiles; the outputs are streamed out once and must not displace it.
   const uint64_t keep_a = ptx::l2_policy_evict_normal(), keep_b = ptx::l2_policy_evict_last(), stream_out = ptx::l2_policy_evict_first();
+  // Reader side of the tile queue: the next tile of this pair, or a number >= n_tiles when there is none (also after
+  // a timeout).
+  int tq_i = 0;     // tiles this thread has taken so far
+  auto next_tile = [&]() -> int {
+    const uint32_t want = (uint32_t)tq_i + 1u, addr = tq_slot(tq_i);
+    ++tq_i;
+    uint32_t seq, v;
+    ptx::ld_shared_volatile_v2(addr, seq, v);
+    if (seq == want) return (int)v;
+    const uint64_t t0 = ptx::globaltimer_ns();
+    for (;;) {
+#pragma unroll 1
+      for (int i = 0; i < 128; ++i) {
+        ptx::ld_shared_volatile_v2(addr, seq, v);
+        if (seq == want) return (int)v;
+      }
+      if (*abort_flag) return 0x7fffffff;
+      if (ptx::globaltimer_ns() - t0 > 4000000000ull) {
+        *abort_flag = 1;
+        return 0x7fffffff;
+      }
+    }
+  };
 
   if (warp == 0) {
     // ===================== TMA producer (both CTAs) =====================
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
-      for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
+      // leader with a tile queue: draws tile numbers and writes them to both CTAs' rings
+      int pq_i = 0;
+      auto publish = [&](int v) {
+        const uint32_t seq = (uint32_t)pq_i + 1u, addr = tq_slot(pq_i);
+        ++pq_i;
+        ptx::st_shared_volatile_v2(addr, seq, (uint32_t)v);
+        ptx::st_shared_cluster_volatile_v2(ptx::map_to_cta(addr, 1), seq, (uint32_t)v);
+        // every pair stops at its first number >= n_tiles, so n_tiles + n_pairs numbers are drawn in all: whoever
+        // holds the last one leaves the counter at zero for the next launch
+        if (v == n_tiles + n_pairs - 1) atomicExch(p.tile_counter, 0u);
+      };
+      const bool draws = DYN && rank == 0;
+      int t = pair_id, t1 = 0x7fffffff;   // this tile and, when drawing, the one after it (already published)
+      if (DYN) {
+        if (draws) {
+          t = (int)atomicAdd(p.tile_counter, 1u);
+          if (t < n_tiles) t1 = (int)atomicAdd(p.tile_counter, 1u);
+          publish(t);
+          if (t < n_tiles) publish(t1);
+        } else {
+          t = next_tile();
+        }
+      }
+      while (t < n_tiles && !*abort_flag) {
+        int t2 = 0x7fffffff;
+        if (draws && t1 < n_tiles) t2 = (int)atomicAdd(p.tile_counter, 1u);   // wanted a whole tile from now
         const Tile ti = decode_tile<MODE>(p, t, rank);
-        for (int ks = 0; ks < ti.num_k; ++ks) {
-          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) break;
+        // a tile with nothing to contract still passes one (empty) stage through the ring, which keeps the producer
+        // within STAGES tiles of the issuer
+        const int steps = ti.num_k > 0 ? ti.num_k : 1;
+        bool ok = true;
+        for (int ks = 0; ks < steps; ++ks) {
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) {
+            ok = false;
+            break;
+          }
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
-          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
-          const uint32_t fb = ptx::map_to_cta(full_bar(s), 0);   // both CTAs' bytes complete on the leader's barrier
-          const int k0 = ks * BK;
-          if (!A_MN) {
-            ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y, keep_a);                       // box {64 k, 128 rows}
+          if (ti.num_k == 0) {
+            if (rank == 0) ptx::mbar_arrive(full_bar(s));
           } else {
-            const int ay = (MODE == MODE_DENSE ? 0 : ti.a_y) + k0;
-            ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay, keep_a);                       // 2 x box {64 m, 64 k}
-            ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay, keep_a);
-          }
-          if (!B_MN) {
-            ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y, keep_b);                       // box {64 k, 128 rows}
-          } else {
-            const int by = (MODE == MODE_DENSE ? 0 : ti.b_y) + k0;
-            ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by, keep_b);                       // 2 x box {64 n, 64 k}
-            ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by, keep_b);
+            if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+            const uint32_t fb = ptx::map_to_cta(full_bar(s), 0);   // both CTAs' bytes complete on the leader's barrier
+            const int k0 = ks * BK;
+            if (!A_MN) {
+              ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y, keep_a);                       // box {64 k, 128 rows}
+            } else {
+              const int ay = (MODE == MODE_DENSE ? 0 : ti.a_y) + k0;
+              ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay, keep_a);                       // 2 x box {64 m, 64 k}
+              ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay, keep_a);
+            }
+            if (!B_MN) {
+              ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y, keep_b);                       // box {64 k, 128 rows}
+            } else {
+              const int by = (MODE == MODE_DENSE ? 0 : ti.b_y) + k0;
+              ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by, keep_b);                       // 2 x box {64 n, 64 k}
+              ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by, keep_b);
+            }
           }
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
           }
+        }
+        if (!ok) break;
+        if (!DYN) {
+          t += n_pairs;
+        } else if (draws) {
+          if (t1 < n_tiles) publish(t2);
+          t = t1;
+          t1 = t2;
+        } else {
+          t = next_tile();
         }
       }
       // every stage release the leader has multicast to this CTA must have landed before the CTA may exit
@@ -311,25 +395,28 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       constexpr uint16_t both = 3;
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
-      for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
+      for (int t = DYN ? next_tile() : pair_id; t < n_tiles && !*abort_flag; t = DYN ? next_tile() : t + n_pairs) {
         const Tile ti = decode_tile<MODE>(p, t, 0);
         if (!ptx::mbar_wait_bounded(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
         bool ok = true;
-        for (int ks = 0; ks < ti.num_k; ++ks) {
+        const int steps = ti.num_k > 0 ? ti.num_k : 1;   // the producer passes one empty stage for a tile without rows
+        for (int ks = 0; ks < steps; ++ks) {
           if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag)) {
             ok = false;
             break;
           }
           ptx::tc_fence_after();
-          const uint32_t sa = smem_base + s * STAGE_BYTES;
-          const uint32_t sb = sa + A_BYTES;
+          if (ti.num_k > 0) {
+            const uint32_t sa = smem_base + s * STAGE_BYTES;
+            const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            const uint64_t da = ptx::make_smem_desc_sw128(sa + kk * a_kadv, a_lbo, a_sbo);
-            const uint64_t db = ptx::make_smem_desc_sw128(sb + kk * b_kadv, b_lbo, b_sbo);
-            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
+            for (int kk = 0; kk < BK / 16; ++kk) {
+              const uint64_t da = ptx::make_smem_desc_sw128(sa + kk * a_kadv, a_lbo, a_sbo);
+              const uint64_t db = ptx::make_smem_desc_sw128(sb + kk * b_kadv, b_lbo, b_sbo);
+              ptx::umma_bf16_pair(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
+            }
           }
           ptx::umma_commit_pair(empty_bar(s), both);  // stage reusable in both CTAs once these MMAs have read it
           if (++s == STAGES) {
@@ -410,7 +497,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int acc = 0;
     uint32_t acc_ph = 0;
     uint32_t flip = 0;                    // staging block the next single-block store uses (they strictly alternate)
-    for (int t = pair_id; t < n_tiles && !*abort_flag; t += n_pairs) {
+    for (int t = DYN ? next_tile() : pair_id; t < n_tiles && !*abort_flag; t = DYN ? next_tile() : t + n_pairs) {
       const Tile ti = decode_tile<MODE>(p, t, rank);
       const bool live = ti.m_valid > 0;    // false: this CTA only lent its half of B to the pair
       uint4 g4[4], u4[4];
@@ -676,6 +763,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.gates = gates;
   p.gate_is_f32 = dm.gate_dtype == GROUTER_GATE_F32;
   p.status = ctx->pp.status;
+  p.tile_counter = ctx->pp.tile_counter;
   Maps m;
   bool ok = true;
   const int grid = ctx->num_sms & ~1;   // whole CTA pairs, one CTA per SM

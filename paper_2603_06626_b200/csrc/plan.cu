@@ -75,7 +75,7 @@ template <typename IdxT>
 __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
                                                                  int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
                                                                  int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
-  extern __shared__ int32_t sm[];  // max(PLAN_WARPS*E, 5*E+5) ints
+  extern __shared__ int32_t sm[];  // plan_hist_smem_ints(E) ints
   __shared__ int s_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
@@ -104,6 +104,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   int32_t* s_pad = sm + 2 * E_tgt + 1;    // [E+1]
   int32_t* s_pair = sm + 3 * E_tgt + 2;   // [E+1] exclusive prefix of 256-row tiles per expert
   int32_t* s_wch = sm + 4 * E_tgt + 3;    // [E+1] exclusive prefix of weight-gradient row chunks per expert
+  int32_t* s_wpos = sm + 5 * E_tgt + 4;   // [2E] list position of each expert's longer / shorter chunks, then [chunk lengths + 1]
   __syncthreads();
   // Exclusive prefix over blocks of every expert's per-block counts (row e of blk_prefix), and the expert totals.
   // Eight lanes share one expert: each sums a contiguous segment of the row with its loads batched eight deep, the
@@ -205,6 +206,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   if (tid == 0) {
     *pp.n_pair_tiles = n_tiles;
     *pp.ticket = 0u;  // ready for the next plan
+    *pp.tile_counter = 0u;  // a grouped GEMM that gave up on a timeout may have left it mid-count
   }
   // expert and first row of every 256-row tile: the last e with s_pair[e] <= t owns tile t
   for (int t = tid; t < n_tiles; t += PLAN_THREADS) {
@@ -217,14 +219,71 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
     pp.pair_row0[t] = row0;
     pp.pair_expert[t] = lo | (row0 + ROW_TILE < s_pad[lo + 1] ? PAIR_VALID2 : 0);
   }
-  // row chunks of the weight-gradient GEMMs: an expert without slots keeps one empty chunk (its gradient is zero-filled)
+  // Row chunks of the weight-gradient GEMMs: an expert without slots keeps one empty chunk (its gradient is zero-filled).
+  // An expert's blocks are cut into n chunks of near-equal size: `rem` chunks of base + 1 blocks, then n - rem of base.
+  // The list is ordered by chunk length, longest first (equal lengths by expert, then by position): the CTA pairs take
+  // tiles round-robin, so neighbours in the list should cost the same or the pairs drift apart and stop sharing
+  // operand rows in L2; the shortest tiles at the end also even out the tail.
   if (tid == 0) *pp.n_wchunks = s_wch[E_tgt];
+  {
+    constexpr int CHUNK_BLOCKS = WGRAD_KCHUNK / ROW_TILE;
+    // chunks of every length, then the first list position of every length (descending)
+    int32_t* s_len = s_wpos + 2 * E_tgt;   // [CHUNK_BLOCKS + 2]
+    for (int i = tid; i <= CHUNK_BLOCKS + 1; i += PLAN_THREADS) s_len[i] = 0;
+    __syncthreads();
+    for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+      const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
+      const int n = s_wch[e + 1] - s_wch[e];
+      const int base = blocks / n, rem = blocks - base * n;
+      if (rem) atomicAdd(&s_len[base + 1], rem);
+      atomicAdd(&s_len[base], n - rem);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int run = 0;
+      for (int l = CHUNK_BLOCKS; l >= 0; --l) {
+        const int c = s_len[l];
+        s_len[l] = run;
+        run += c;
+      }
+    }
+    __syncthreads();
+    // within one length: experts in ascending order.  One warp per length walks the experts 32 at a time.
+    for (int l = warp; l <= CHUNK_BLOCKS; l += PLAN_WARPS) {
+      int run = s_len[l];
+      for (int e0 = 0; e0 < E_tgt; e0 += 32) {
+        const int e = e0 + lane;
+        int cnt = 0, which = -1;
+        if (e < E_tgt) {
+          const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
+          const int n = s_wch[e + 1] - s_wch[e];
+          const int base = blocks / n, rem = blocks - base * n;
+          if (rem && base + 1 == l) {
+            cnt = rem;
+            which = 0;
+          } else if (base == l) {
+            cnt = n - rem;
+            which = 1;
+          }
+        }
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        if (which >= 0) s_wpos[which * E_tgt + e] = run + incl - cnt;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+      }
+    }
+    __syncthreads();
+  }
   for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
     const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
     const int n = s_wch[e + 1] - s_wch[e];
-    const int base = blocks / n, rem = blocks - base * n;   // chunks of near-equal size: the first `rem` hold one block more
+    const int base = blocks / n, rem = blocks - base * n;
     for (int c = 0; c < n; ++c) {
-      const int i = s_wch[e] + c;
+      const int i = c < rem ? s_wpos[e] + c : s_wpos[E_tgt + e] + (c - rem);
       pp.wchunk_expert[i] = e | (n > 1 ? WCHUNK_SPLIT : 0);
       pp.wchunk_row0[i] = s_pad[e] + (c * base + min(c, rem)) * ROW_TILE;
       int rows = (base + (c < rem ? 1 : 0)) * ROW_TILE;
@@ -294,6 +353,12 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_permute_kernel(const IdxT* 
   }
 }
 
+// per-warp histograms while counting; the last block's scans and chunk ordering afterwards
+static int plan_hist_smem_ints(int E) {
+  const int a = PLAN_WARPS * E, b = 7 * E + 4 + WGRAD_KCHUNK / ROW_TILE + 2;
+  return a > b ? a : b;
+}
+
 template <typename IdxT>
 static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, const int32_t* fold_map, int32_t* counts,
                                  int32_t* offsets, int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
@@ -301,7 +366,7 @@ static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, c
   const int R = (int)ctx->R, E = dm.E_tgt;
   const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
   if (phase == 0) {
-    const size_t sm1 = sizeof(int32_t) * (size_t)((PLAN_WARPS * E > 5 * E + 5) ? PLAN_WARPS * E : 5 * E + 5);
+    const size_t sm1 = sizeof(int32_t) * (size_t)plan_hist_smem_ints(E);
     plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
   } else {
     const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
@@ -423,6 +488,7 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.pp.pad_begin = base + NA_PAD_BEGIN;
   c.pp.n_pair_tiles = base + NA_N_TILES;
   c.pp.ticket = reinterpret_cast<unsigned int*>(base + NA_TICKET);
+  c.pp.tile_counter = c.pp.ticket + 4;
   c.pp.status = status ? status : base + NA_STATUS;
   c.pp.pair_row0 = base + NA_PAIR_ROW0;
   c.pp.pair_expert = base + NA_PAIR_EXPERT;

@@ -88,6 +88,20 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   }
 }
 
+// ---------------- 8-byte words polled across the CTA pair ----------------
+// A volatile 8-byte store / load of an aligned shared-memory word is a single access: a reader sees the old pair or
+// the new pair, never a mix.  The cluster form writes the shared memory of any CTA of the cluster (address from
+// map_to_cta).
+__device__ __forceinline__ void st_shared_volatile_v2(uint32_t addr, uint32_t a, uint32_t b) {
+  asm volatile("st.volatile.shared.v2.u32 [%0], {%1, %2};" ::"r"(addr), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ void st_shared_cluster_volatile_v2(uint32_t cluster_addr, uint32_t a, uint32_t b) {
+  asm volatile("st.volatile.shared::cluster.v2.u32 [%0], {%1, %2};" ::"r"(cluster_addr), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ void ld_shared_volatile_v2(uint32_t addr, uint32_t& a, uint32_t& b) {
+  asm volatile("ld.volatile.shared.v2.u32 {%0, %1}, [%2];" : "=r"(a), "=r"(b) : "r"(addr) : "memory");
+}
+
 // ---------------- L2 eviction policies for TMA copies ----------------
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {   // streamed once: do not displace what is reused
   uint64_t p;
