@@ -158,7 +158,16 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->R = (int64_t)dims->T * dims->k;
   c->R_pad_max = r_pad_max(*dims);
   c->max_m_tiles = (int)(c->R_pad_max / ROW_TILE);
-  c->max_wchunks = dims->E_tgt + (int)(c->R_pad_max / WGRAD_KCHUNK) + 1;
+  {
+    // Chunk length of the weight gradients: as long as possible, but short enough that the smaller of the two
+    // gradients (d x ffn per expert) still yields about four tiles per CTA pair over the whole batch.
+    const int64_t tiles_d = (int64_t)((dims->d + 255) / 256) * ((dims->ffn + 255) / 256);
+    const int64_t want = c->R_pad_max * tiles_d / (4 * (int64_t)(sms > 1 ? sms / 2 : 1));
+    int chunk = WGRAD_KCHUNK_MAX;
+    while (chunk > WGRAD_KCHUNK_MIN && chunk > want) chunk >>= 1;
+    c->pp.wgrad_chunk_blocks = chunk / ROW_TILE;
+    c->max_wchunks = dims->E_tgt + (int)(c->R_pad_max / chunk) + 1;
+  }
   c->geom = plan_geom(c->R);
   c->planned = c->forwarded = false;
   c->ev_start = c->ev_stop = nullptr;

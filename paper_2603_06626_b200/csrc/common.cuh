@@ -15,9 +15,11 @@ constexpr int STATUS_TIMEOUT = 2;
 
 constexpr int ROW_TILE = 128;        // rows one CTA owns in a GEMM tile; expert segments are padded to it
 constexpr int PAIR_VALID2 = 1 << 30; // flag in PaddedPlan::pair_expert
-// The weight-gradient GEMMs contract over an expert's rows in chunks of at most this many (padded) rows, so that
-// the operand rows of one chunk stay in L2 while every output tile of the expert reads them.
-constexpr int WGRAD_KCHUNK = 4096;
+// The weight-gradient GEMMs contract over an expert's rows in chunks of at most `wgrad_chunk_blocks` row tiles; an expert
+// with several chunks has its gradient summed from partial tiles.  Long chunks mean few partial sums; short chunks give
+// the CTA pairs enough tiles when the output matrices are small.  The context picks a power of two between these bounds.
+constexpr int WGRAD_KCHUNK_MIN = 1024, WGRAD_KCHUNK_MAX = 16384;
+constexpr int WGRAD_LEN_BUCKETS = 32;   // the chunk list is ordered by chunk length in this many classes
 constexpr int WCHUNK_SPLIT = 1 << 30; // flag in PaddedPlan::wchunk_expert: the expert has several chunks
 constexpr int PLAN_THREADS = 256;    // 8 warps per plan block
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
@@ -60,6 +62,7 @@ struct PaddedPlan {
   int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows
   int32_t* blk_prefix;    // [E_tgt * nblk] per-block histogram, then exclusive prefix over blocks
   unsigned int* ticket;   // [1] last-block-done counter
+  int wgrad_chunk_blocks;       // longest weight-gradient chunk, in row tiles
   unsigned int* tile_counter;   // [1] next tile of the running grouped GEMM; zero between launches
   int32_t* status;        // [1] sticky status bits
 };
@@ -72,7 +75,7 @@ struct grouter_ctx {
   int64_t R;
   int64_t R_pad_max;      // round_up(R,128) + 128*E_tgt
   int max_m_tiles;
-  int max_wchunks;        // E_tgt + R_pad_max / WGRAD_KCHUNK + 1
+  int max_wchunks;        // E_tgt + R_pad_max / (chunk rows) + 1
   grouter::PlanGeom geom;
   grouter::PaddedPlan pp;
   void* d_block;          // one allocation backing pp

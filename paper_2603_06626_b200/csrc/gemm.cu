@@ -74,7 +74,8 @@ struct GemmParams {
 struct Tile {     // one CTA's share of a pair tile
   int a_x, a_y;   // TMA coordinates of this CTA's A rows at k-step 0
   int b_x, b_y;   // ... and of this CTA's half of B
-  int num_k;
+  int num_k;      // k-steps that contribute to the result
+  int steps;      // k-steps that pass through the operand ring: max(num_k, 1)
   int row0, col0; // origin of this CTA's 128 x 256 output block within the output matrix of this problem
   int e;
   int m_valid, n_valid;   // m_valid <= 0: this CTA's rows are not part of the problem (it still feeds its B half)
@@ -153,10 +154,12 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
     ti.m_valid = min(BM, p.M - ti.row0);
     ti.n_valid = min(BN, p.N - ti.col0);
     ti.a_x = ti.row0;   // both operands MN-major: x runs along M/N, y along the expert's rows
-    ti.a_y = k0;
     ti.b_x = ti.col0 + rank * BNH;
-    ti.b_y = k0;
     ti.num_k = (k1 - k0) / BK;
+    // An expert without rows still sends one k-step through the pipeline, so that every tile is paced by the same
+    // barriers: its boxes lie beyond the last row, where TMA fills zeros without touching memory, and the epilogue
+    // ignores the accumulator.
+    ti.a_y = ti.b_y = ti.num_k > 0 ? k0 : (int)p.R_pad_max;
   } else {  // DENSE
     const int mt = t / p.tiles_n, nt = t - mt * p.tiles_n;
     ti.e = 0;
@@ -170,6 +173,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
     ti.b_y = ti.col0 + rank * BNH;
     ti.num_k = (p.K + BK - 1) / BK;
   }
+  ti.steps = ti.num_k > 0 ? ti.num_k : 1;
   return ti;
 }
 
@@ -325,37 +329,30 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int t2 = 0x7fffffff;
         if (draws && t1 < n_tiles) t2 = (int)atomicAdd(p.tile_counter, 1u);   // wanted a whole tile from now
         const Tile ti = decode_tile<MODE>(p, t, rank);
-        // a tile with nothing to contract still passes one (empty) stage through the ring, which keeps the producer
-        // within STAGES tiles of the issuer
-        const int steps = ti.num_k > 0 ? ti.num_k : 1;
         bool ok = true;
-        for (int ks = 0; ks < steps; ++ks) {
+        for (int ks = 0; ks < ti.steps; ++ks) {
           if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) {
             ok = false;
             break;
           }
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
-          if (ti.num_k == 0) {
-            if (rank == 0) ptx::mbar_arrive(full_bar(s));
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+          const uint32_t fb = ptx::map_to_cta(full_bar(s), 0);   // both CTAs' bytes complete on the leader's barrier
+          const int k0 = ks * BK;
+          if (!A_MN) {
+            ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y, keep_a);                       // box {64 k, 128 rows}
           } else {
-            if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
-            const uint32_t fb = ptx::map_to_cta(full_bar(s), 0);   // both CTAs' bytes complete on the leader's barrier
-            const int k0 = ks * BK;
-            if (!A_MN) {
-              ptx::tma_load_2d_pair(sa, &tmA, fb, k0, ti.a_y, keep_a);                       // box {64 k, 128 rows}
-            } else {
-              const int ay = (MODE == MODE_DENSE ? 0 : ti.a_y) + k0;
-              ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay, keep_a);                       // 2 x box {64 m, 64 k}
-              ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay, keep_a);
-            }
-            if (!B_MN) {
-              ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y, keep_b);                       // box {64 k, 128 rows}
-            } else {
-              const int by = (MODE == MODE_DENSE ? 0 : ti.b_y) + k0;
-              ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by, keep_b);                       // 2 x box {64 n, 64 k}
-              ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by, keep_b);
-            }
+            const int ay = (MODE == MODE_DENSE ? 0 : ti.a_y) + k0;
+            ptx::tma_load_2d_pair(sa, &tmA, fb, ti.a_x, ay, keep_a);                       // 2 x box {64 m, 64 k}
+            ptx::tma_load_2d_pair(sa + ATOM_BYTES, &tmA, fb, ti.a_x + 64, ay, keep_a);
+          }
+          if (!B_MN) {
+            ptx::tma_load_2d_pair(sb, &tmB, fb, k0, ti.b_y, keep_b);                       // box {64 k, 128 rows}
+          } else {
+            const int by = (MODE == MODE_DENSE ? 0 : ti.b_y) + k0;
+            ptx::tma_load_2d_pair(sb, &tmB, fb, ti.b_x, by, keep_b);                       // 2 x box {64 n, 64 k}
+            ptx::tma_load_2d_pair(sb + ATOM_BYTES, &tmB, fb, ti.b_x + 64, by, keep_b);
           }
           if (++s == STAGES) {
             s = 0;
@@ -401,22 +398,19 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
         bool ok = true;
-        const int steps = ti.num_k > 0 ? ti.num_k : 1;   // the producer passes one empty stage for a tile without rows
-        for (int ks = 0; ks < steps; ++ks) {
+        for (int ks = 0; ks < ti.steps; ++ks) {
           if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag)) {
             ok = false;
             break;
           }
           ptx::tc_fence_after();
-          if (ti.num_k > 0) {
-            const uint32_t sa = smem_base + s * STAGE_BYTES;
-            const uint32_t sb = sa + A_BYTES;
+          const uint32_t sa = smem_base + s * STAGE_BYTES;
+          const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk) {
-              const uint64_t da = ptx::make_smem_desc_sw128(sa + kk * a_kadv, a_lbo, a_sbo);
-              const uint64_t db = ptx::make_smem_desc_sw128(sb + kk * b_kadv, b_lbo, b_sbo);
-              ptx::umma_bf16_pair(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
-            }
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            const uint64_t da = ptx::make_smem_desc_sw128(sa + kk * a_kadv, a_lbo, a_sbo);
+            const uint64_t db = ptx::make_smem_desc_sw128(sb + kk * b_kadv, b_lbo, b_sbo);
+            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
           }
           ptx::umma_commit_pair(empty_bar(s), both);  // stage reusable in both CTAs once these MMAs have read it
           if (++s == STAGES) {
@@ -425,12 +419,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
         if (!ok) break;
-        if (ti.num_k > 0) {
-          ptx::umma_commit_pair(tfull_bar(acc), both);
-        } else {                                      // nothing to contract: the epilogues write zeros
-          ptx::mbar_arrive(tfull_bar(acc));
-          ptx::mbar_arrive_cluster(ptx::map_to_cta(tfull_bar(acc), 1));
-        }
+        ptx::umma_commit_pair(tfull_bar(acc), both);
         if (++acc == 2) {
           acc = 0;
           acc_ph ^= 1u;

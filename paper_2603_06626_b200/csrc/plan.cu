@@ -149,8 +149,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   if (warp == 0) {
     const int per = (E_tgt + 31) / 32;
     const int e0 = min(lane * per, E_tgt), e1 = min(e0 + per, E_tgt);
-    constexpr int CHUNK_BLOCKS = WGRAD_KCHUNK / ROW_TILE;
-    auto chunks_of = [](int blocks) { return blocks == 0 ? 1 : (blocks + CHUNK_BLOCKS - 1) / CHUNK_BLOCKS; };
+    const int chunk_blocks = pp.wgrad_chunk_blocks;
+    auto chunks_of = [chunk_blocks](int blocks) { return blocks == 0 ? 1 : (blocks + chunk_blocks - 1) / chunk_blocks; };
     int sum = 0, psum = 0, tsum = 0, wsum = 0;
     for (int e = e0; e < e1; ++e) {
       const int blocks = (s_cnt[e] + ROW_TILE - 1) / ROW_TILE;
@@ -221,58 +221,56 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
   }
   // Row chunks of the weight-gradient GEMMs: an expert without slots keeps one empty chunk (its gradient is zero-filled).
   // An expert's blocks are cut into n chunks of near-equal size: `rem` chunks of base + 1 blocks, then n - rem of base.
-  // The list is ordered by chunk length, longest first (equal lengths by expert, then by position): the CTA pairs take
-  // tiles round-robin, so neighbours in the list should cost the same or the pairs drift apart and stop sharing
-  // operand rows in L2; the shortest tiles at the end also even out the tail.
+  // The list is ordered by chunk length, longest first, in WGRAD_LEN_BUCKETS classes of length (within a class by
+  // expert, then by position): tiles of similar cost are neighbours, and the shortest tiles at the end even out the tail.
   if (tid == 0) *pp.n_wchunks = s_wch[E_tgt];
   {
-    constexpr int CHUNK_BLOCKS = WGRAD_KCHUNK / ROW_TILE;
-    // chunks of every length, then the first list position of every length (descending)
-    int32_t* s_len = s_wpos + 2 * E_tgt;   // [CHUNK_BLOCKS + 2]
-    for (int i = tid; i <= CHUNK_BLOCKS + 1; i += PLAN_THREADS) s_len[i] = 0;
+    const int chunk_blocks = pp.wgrad_chunk_blocks;
+    auto len_class = [chunk_blocks](int blocks) { return (blocks * WGRAD_LEN_BUCKETS + chunk_blocks - 1) / chunk_blocks; };   // 0 .. BUCKETS
+    // chunks of every class, then the first list position of every class (descending)
+    int32_t* s_len = s_wpos + 2 * E_tgt;   // [WGRAD_LEN_BUCKETS + 1]
+    for (int i = tid; i <= WGRAD_LEN_BUCKETS; i += PLAN_THREADS) s_len[i] = 0;
     __syncthreads();
     for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
       const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
       const int n = s_wch[e + 1] - s_wch[e];
       const int base = blocks / n, rem = blocks - base * n;
-      if (rem) atomicAdd(&s_len[base + 1], rem);
-      atomicAdd(&s_len[base], n - rem);
+      if (rem) atomicAdd(&s_len[len_class(base + 1)], rem);
+      atomicAdd(&s_len[len_class(base)], n - rem);
     }
     __syncthreads();
     if (tid == 0) {
       int run = 0;
-      for (int l = CHUNK_BLOCKS; l >= 0; --l) {
+      for (int l = WGRAD_LEN_BUCKETS; l >= 0; --l) {
         const int c = s_len[l];
         s_len[l] = run;
         run += c;
       }
     }
     __syncthreads();
-    // within one length: experts in ascending order.  One warp per length walks the experts 32 at a time.
-    for (int l = warp; l <= CHUNK_BLOCKS; l += PLAN_WARPS) {
+    // within one class: experts in ascending order, an expert's longer chunks before its shorter ones.  One warp per
+    // class walks the experts 32 at a time.
+    for (int l = warp; l <= WGRAD_LEN_BUCKETS; l += PLAN_WARPS) {
       int run = s_len[l];
       for (int e0 = 0; e0 < E_tgt; e0 += 32) {
         const int e = e0 + lane;
-        int cnt = 0, which = -1;
+        int c0 = 0, c1 = 0;    // chunks of the expert's two lengths that fall into class l
         if (e < E_tgt) {
           const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
           const int n = s_wch[e + 1] - s_wch[e];
           const int base = blocks / n, rem = blocks - base * n;
-          if (rem && base + 1 == l) {
-            cnt = rem;
-            which = 0;
-          } else if (base == l) {
-            cnt = n - rem;
-            which = 1;
-          }
+          if (rem && len_class(base + 1) == l) c0 = rem;
+          if (len_class(base) == l) c1 = n - rem;
         }
-        int incl = cnt;
+        int incl = c0 + c1;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           const int v = __shfl_up_sync(0xffffffffu, incl, o);
           if (lane >= o) incl += v;
         }
-        if (which >= 0) s_wpos[which * E_tgt + e] = run + incl - cnt;
+        const int first = run + incl - (c0 + c1);
+        if (c0) s_wpos[e] = first;
+        if (c1) s_wpos[E_tgt + e] = first + c0;
         run += __shfl_sync(0xffffffffu, incl, 31);
       }
     }
@@ -355,7 +353,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_permute_kernel(const IdxT* 
 
 // per-warp histograms while counting; the last block's scans and chunk ordering afterwards
 static int plan_hist_smem_ints(int E) {
-  const int a = PLAN_WARPS * E, b = 7 * E + 4 + WGRAD_KCHUNK / ROW_TILE + 2;
+  const int a = PLAN_WARPS * E, b = 7 * E + 4 + WGRAD_LEN_BUCKETS + 2;
   return a > b ? a : b;
 }
 
@@ -416,7 +414,7 @@ constexpr int NA_TICKET = NA_N_TILES + 64;                            // [1]
 constexpr int NA_STATUS = NA_TICKET + 64;                             // [1] used when the caller passes no status word
 constexpr int NA_PAIR_ROW0 = NA_STATUS + 64;                          // [rows/128]
 constexpr int NA_PAIR_EXPERT = NA_PAIR_ROW0 + NOALLOC_MAX_ROWS / ROW_TILE;     // [rows/128]
-constexpr int NOALLOC_MAX_WCHUNKS = (NOALLOC_MAX_E + NOALLOC_MAX_ROWS / WGRAD_KCHUNK + 1 + 63) / 64 * 64;
+constexpr int NOALLOC_MAX_WCHUNKS = (NOALLOC_MAX_E + NOALLOC_MAX_ROWS / WGRAD_KCHUNK_MAX + 1 + 63) / 64 * 64;
 constexpr int NA_WCHUNK_EXPERT = NA_PAIR_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE; // [chunks]
 constexpr int NA_WCHUNK_ROW0 = NA_WCHUNK_EXPERT + NOALLOC_MAX_WCHUNKS;         // [chunks]
 constexpr int NA_WCHUNK_ROWS = NA_WCHUNK_ROW0 + NOALLOC_MAX_WCHUNKS;           // [chunks]
@@ -489,6 +487,7 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.pp.n_pair_tiles = base + NA_N_TILES;
   c.pp.ticket = reinterpret_cast<unsigned int*>(base + NA_TICKET);
   c.pp.tile_counter = c.pp.ticket + 4;
+  c.pp.wgrad_chunk_blocks = WGRAD_KCHUNK_MAX / ROW_TILE;   // the chunk list is scratch here: fewest entries
   c.pp.status = status ? status : base + NA_STATUS;
   c.pp.pair_row0 = base + NA_PAIR_ROW0;
   c.pp.pair_expert = base + NA_PAIR_EXPERT;

@@ -57,5 +57,8 @@ def test_step_host_matches_device_calls_with_steps_in_flight(name, n_steps):
     layer.check_status()
     h = host[-1]
     assert torch.equal(h["Y"], expected[-1][0]) and torch.equal(h["dX"], expected[-1][1]) and torch.equal(h["dg"], expected[-1][2])
-    assert torch.equal(dW_gu.cpu(), expected[-1][3]) and torch.equal(dW_d.cpu(), expected[-1][4])
+    # an expert whose rows span several chunks has its gradient summed from partial tiles with fp32 atomics, whose order
+    # is not fixed: equal up to that reordering
+    for got, want in ((dW_gu.cpu(), expected[-1][3]), (dW_d.cpu(), expected[-1][4])):
+        assert (got - want).double().norm() <= 1e-6 * want.double().norm()
     layer.close()
