@@ -156,6 +156,7 @@ def test_large_sampled():
     (640, 384, 344, 128, 8, {}),                   # another: more experts than tiles per expert
     (900, 512, 704, 64, 6, {"load": "zipf", "zipf_s": 1.3, "n_dead": 7}),
     (512, 1024, 384, 128, 8, {}),
+    (192, 256, 256, 128, 2, {"n_dead": 112}),      # long runs of experts without rows: tiles that contract nothing
 ])
 def test_edge_shapes_full_parity(T, d, F, E, k, kw):
     w = synth.custom_workload("edge", T=T, d=d, ffn=F, E=E, k=k, seed=T + d, **kw)
