@@ -178,13 +178,13 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def kernel_work(w: synth.Workload, counts: np.ndarray):
+def kernel_work(w: synth.Workload, counts: np.ndarray, chunk_rows: int):
     """Algorithmic work per launch: FLOPs over valid routed rows only (padding earns nothing) for the
     GEMMs; bytes (T + R) * d * 2 for the row movers; plan: ids read, two permutations written; the zero-fill
-    writes the fp32 gradients of the experts whose rows are contracted in several chunks (more than 4096
-    padded rows)."""
+    writes the fp32 gradients of the experts whose rows are contracted in several chunks (more than
+    `chunk_rows` padded rows)."""
     R, d, F, T = w.R, w.d, w.ffn, w.T
-    n_split = int((((counts + 127) // 128) * 128 > 4096).sum())
+    n_split = int((((counts + 127) // 128) * 128 > chunk_rows).sum())
     dF = 2.0 * R * d * F
     idb = 1 if w.E_src <= 256 else 4
     return {
@@ -467,7 +467,7 @@ def main():
 
     # ---- roofline of the dominant kernel, and the per-kernel table ----
     peaks, peak_src = load_peaks()
-    work = kernel_work(w, layer.counts.cpu().numpy().astype(np.int64))
+    work = kernel_work(w, layer.counts.cpu().numpy().astype(np.int64), layer.wgrad_chunk_rows())
     kernels = {}
     for name, (ms, n) in per_kernel.items():
         if n == 0:

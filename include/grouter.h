@@ -195,13 +195,19 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
  *   dW_gu  [E_tgt, 2*ffn, d] f32 out  dW_d   [E_tgt, d, ffn] f32 out
  *   dgates [T,k] f32 out: dgates[t,j] = <dY[t,:], f_{e(t,j)}(X[t,:])> (gates are leaf inputs)
  * Experts that received no slot get exact zeros in dW_* (with GROUTER_FLAG_ACCUMULATE_DW every expert's gradient is
- * added to what dW_* holds, and such experts are left as they are).  An expert with more than 4096 rows is contracted in
- * chunks of rows that are added into its gradient in no fixed order, so its dW_* may differ in the last bits
- * from run to run; everything else (Y, dX, dgates, dW_* of smaller experts) is bit-reproducible.  Uses the workspace
+ * added to what dW_* holds, and such experts are left as they are).  An expert with more than
+ * grouter_wgrad_chunk_rows(ctx) rows is contracted in chunks of rows that are added into its gradient in no fixed order,
+ * so its dW_* may differ in the last bits from run to run; everything else (Y, dX, dgates, dW_* of smaller experts) is bit-reproducible.  Uses the workspace
  * contents left by the matching grouter_moe_fwd (else INVALID_STATE). */
 int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void* gates, const void* W_gu,
                     const void* W_d, void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace,
                     void* stream);
+
+/* Longest run of an expert's rows that the weight-gradient products of grouter_moe_bwd contract in one piece (host
+ * only; a power of two between 1024 and 16384 fixed at grouter_create from the dims and the device's SM count: as long
+ * as possible, shorter when the per-expert gradient matrices are too small to keep every SM busy otherwise).  The
+ * paper has no counterpart: it is a scheduling parameter of this implementation.  Returns 0 for a null context. */
+int32_t grouter_wgrad_chunk_rows(const grouter_ctx* ctx);
 
 /* One whole step from HOST buffers: uploads idx, gates, X, dY, runs plan, fwd and bwd on `stream`, and downloads
  * Y, dX, dgates.  Weights, weight gradients and fold_map stay on the device.  The copies run on two streams the

@@ -448,6 +448,8 @@ int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t
   return GROUTER_OK;
 }
 
+int32_t grouter_wgrad_chunk_rows(const grouter_ctx* ctx) { return ctx ? ctx->pp.wgrad_chunk_blocks * grouter::ROW_TILE : 0; }
+
 int grouter_dense_gemm(const void* A, int a_mn_major, const void* B, int b_mn_major, float* C, int32_t M, int32_t N, int32_t K,
                        int32_t* status, void* stream) {
   if (!A || !B || !C || !status || M < 1 || N < 1 || K < 1) return GROUTER_ERR_INVALID_ARG;
