@@ -24,7 +24,10 @@
 // Operands may be K-major (rows of the stored matrix run along K) or MN-major (rows run along M/N); both are
 // described to the MMA by shared-memory descriptors, so no operand is ever transposed in memory.
 //
-// Every mbarrier wait is bounded; on give-up the CTA raises an abort flag, ORs STATUS_TIMEOUT into the status
+// Tiles are handed out by a grid-wide counter (all products but DENSE): a pair takes the next tile of the list when it
+// is ready for one, so the pairs always work on neighbouring tiles and the operand rows they share are in L2 together.
+//
+// Every wait (mbarriers, tile queue) is bounded; on give-up the CTA raises an abort flag, ORs STATUS_TIMEOUT into the status
 // word, leaves its loops, and the pair meets at a cluster barrier before freeing TMEM and exiting.
 #include "common.cuh"
 #include "ptx.cuh"
