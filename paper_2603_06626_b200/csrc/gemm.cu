@@ -212,7 +212,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stage_base = smem_base + STAGES * STAGE_BYTES;          // epilogue staging, 2 x 4 KB per warp
   const uint32_t bar_base = stage_base + EPI_WARPS * 2 * EPI_STAGE_BYTES;
-  // barriers (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+  // barriers (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]; then the tile queue's slots
   //   full[s]       leader only: one arrival (leader's producer, with the byte count of BOTH CTAs' loads)
   //   empty[s]      each CTA: one arrival per round, delivered to both CTAs by the leader's multicast commit
   //   tmem_full[a]  each CTA: one arrival per tile, delivered to both CTAs by the leader's multicast commit

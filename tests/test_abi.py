@@ -38,3 +38,4 @@ def test_host_only_calls_need_no_gpu():
     assert n >= rows * (3 * 256 + 5 * 512) * 2     # Xp, O, dYp [rows,d]; G, U, H, dG|dU [rows,F]
     bad = binding.GrouterDims(512, 250, 512, 8, 8, 2, 0, 0, 0)
     assert lib.grouter_workspace_bytes(ctypes.byref(bad)) == 0
+    assert lib.grouter_wgrad_chunk_rows(None) == 0   # null context

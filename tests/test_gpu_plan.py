@@ -132,3 +132,16 @@ def test_kernel_timing_records_and_idle_gap():
         layer.timing_gap(-1)
     assert layer.status() == 0
     layer.close()
+
+
+def test_weight_gradient_chunk_length_follows_the_problem_size():
+    """Long chunks (few partial sums) when the batch gives every CTA pair tiles anyway, short ones for small problems."""
+    from paper_2603_06626_b200 import binding
+    got = {}
+    for name in ("tiny", "small", "skewed", "large"):
+        w = synth.WORKLOADS[name]
+        layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt)
+        got[name] = layer.wgrad_chunk_rows()
+        layer.close()
+    assert all(1024 <= v <= 16384 and v & (v - 1) == 0 for v in got.values()), got
+    assert got["tiny"] == 1024 and got["large"] == 16384 and got["small"] <= got["skewed"], got
