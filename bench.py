@@ -390,11 +390,16 @@ def main():
     layer.timing_enable(len(binding.KERNEL_SLOTS) * args.steps)
     wall0 = time.time()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps - 1)]   # between steps: median / best step
     ev0.record()
-    for _ in range(args.steps):
+    for i in range(args.steps):
         step()
+        if i < args.steps - 1:
+            marks[i].record()
     ev1.record()
     torch.cuda.synchronize()
+    edges = [ev0] + marks + [ev1]
+    step_ms = sorted(edges[i].elapsed_time(edges[i + 1]) for i in range(args.steps))
     wall1 = time.time()
     barrier()
     ms_total = ev0.elapsed_time(ev1)
@@ -518,7 +523,7 @@ def main():
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "ms_per_step": ms_step, "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_best": step_ms[0], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(base, world), "clocks": clocks,
         "gpu_launches": int(sum(v[1] for v in per_kernel.values())), "roofline": roofline, "kernels": kernels, "gemm_summary": summary, "plan": plan,
         "load_stats": synth.load_stats(li.idx, li.fold_map, w.E_tgt),
