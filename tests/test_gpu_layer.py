@@ -240,3 +240,46 @@ def test_accumulate_dw_over_micro_batches():
     layer.close()
     with pytest.raises(binding.GrouterError):
         binding.GrouterLayer(64, 64, 64, 4, 2, flags=4)      # unknown flag bit
+
+
+def test_whole_step_replays_from_a_cuda_graph():
+    """plan + fwd + bwd only enqueue kernels on the caller's stream (no allocation, no synchronisation), so a step can be
+    captured once and replayed; the replay is bit-identical for everything that is reproducible."""
+    from paper_2603_06626_b200 import binding
+    w = synth.WORKLOADS["tiny"]
+    li = synth.make_layer_inputs(w)
+    idx, gates, X, dY = to_dev(li.idx), bits_to_bf16(li.gates), bits_to_bf16(li.X), bits_to_bf16(li.dY)
+    W_gu, W_d = bits_to_bf16(li.W_gu), bits_to_bf16(li.W_d)
+    layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt)
+    Y, dX = torch.empty_like(X), torch.empty_like(X)
+    dg = torch.empty(w.T, w.k, device=X.device, dtype=torch.float32)
+    dW_gu = torch.empty(W_gu.shape, device=X.device, dtype=torch.float32)
+    dW_d = torch.empty(W_d.shape, device=X.device, dtype=torch.float32)
+
+    def step():
+        layer.plan(idx)
+        layer.forward(X, gates, W_gu, W_d, Y)
+        layer.backward(dY, X, gates, W_gu, W_d, dX, dW_gu, dW_d, dg)
+
+    step()
+    layer.check_status()
+    want = [t.clone() for t in (Y.view(torch.int16), dX.view(torch.int16), dg, dW_gu, dW_d)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):      # warm-up on a side stream, as capture requires
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for t in (Y, dX, dg, dW_gu, dW_d):
+        t.zero_()
+    for _ in range(3):
+        graph.replay()
+    layer.check_status()
+    got = (Y.view(torch.int16), dX.view(torch.int16), dg, dW_gu, dW_d)
+    for g, x in zip(got[:3], want[:3]):
+        assert torch.equal(g, x)
+    for g, x in zip(got[3:], want[3:]):      # experts cut into several chunks are summed with atomics
+        assert (g - x).double().norm() <= 1e-6 * x.double().norm()
+    layer.close()
