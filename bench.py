@@ -423,6 +423,25 @@ def main():
         layer.timing_gap(0)
         layer.check_status()
 
+    # ---- where the issuers' cycles go (a few steps with the accounting on; not part of any timed number) ----
+    gemm_cycles = None
+    if world == 1 and not args.no_isolated:
+        layer.gemm_cycles_enable(True)
+        step()
+        layer.gemm_cycles_read()
+        for _ in range(5):
+            step()
+        raw = layer.gemm_cycles_read()
+        layer.gemm_cycles_enable(False)
+        layer.check_status()
+        gemm_cycles = {}
+        for name, c in raw.items():
+            if c["k_steps"] > 0 and c["cycles"] > 0:
+                gemm_cycles[name] = {"cycles_per_k_step": c["cycles"] / c["k_steps"], "tensor_core_cycles_per_k_step": 512,
+                                     "wait_operands_frac": c["wait_operands"] / c["cycles"],
+                                     "wait_accumulator_frac": c["wait_accumulator"] / c["cycles"],
+                                     "tiles_per_pair_per_launch": c["tiles"] / 5.0 / max(1, torch.cuda.get_device_properties(dev).multi_processor_count // 2)}
+
     # ---- end to end: host buffers in, host results out, every step ----
     e2e = None
     if not args.no_e2e:
@@ -526,6 +545,7 @@ def main():
         "ms_per_step": ms_step, "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_best": step_ms[0], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(base, world), "clocks": clocks,
         "gpu_launches": int(sum(v[1] for v in per_kernel.values())), "roofline": roofline, "kernels": kernels, "gemm_summary": summary, "plan": plan,
+        "gemm_cycles": gemm_cycles,
         "load_stats": synth.load_stats(li.idx, li.fold_map, w.E_tgt),
     }
     if e2e is not None:

@@ -249,6 +249,16 @@ int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records);
  * every timed kernel, so that each kernel is measured on a GPU that is not already at its power cap: the figure to
  * hold against a burst peak, where the back-to-back figure belongs with a sustained peak. */
 int grouter_timing_gap(grouter_ctx* ctx, int32_t microseconds);
+
+/* Measurement aid with no counterpart in the paper: where the tensor-core issuers' cycles go.  While enabled (on != 0;
+ * off by default), the one MMA-issuing thread of every CTA pair of every grouped GEMM of fwd/bwd adds to five device
+ * counters per GEMM: [0] its SM cycles from first tile to last, [1] of these the cycles spent waiting for operand stages
+ * to arrive in shared memory, [2] the cycles spent waiting for a free accumulator (epilogue behind), [3] tiles, [4] k-steps
+ * (256 x 256 x 64 each; the tensor cores need 512 cycles for one).  grouter_gemm_cycles_read copies the sums since the
+ * last read into counters (HOST array of 6 x 5 values, GEMMs in the order up, down, dH, dX, wgrad_down, wgrad_gate_up),
+ * zeroes them and synchronises `stream`.  The accounting costs a few clock reads per k-step: leave it off when timing. */
+int grouter_gemm_cycles_enable(grouter_ctx* ctx, int32_t on);
+int grouter_gemm_cycles_read(grouter_ctx* ctx, void* stream, uint64_t* counters);
 int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t* launches);
 
 /* Component check of the tensor-core core used by every grouped GEMM (no

@@ -22,7 +22,7 @@ GATE_BF16, GATE_F32 = 0, 1
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
-           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows"]
+           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW"]
 
@@ -89,6 +89,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_timing_enable.restype = ctypes.c_int
     lib.grouter_timing_gap.argtypes = [vp, ctypes.c_int32]
     lib.grouter_timing_gap.restype = ctypes.c_int
+    lib.grouter_gemm_cycles_enable.argtypes = [vp, ctypes.c_int32]
+    lib.grouter_gemm_cycles_enable.restype = ctypes.c_int
+    lib.grouter_gemm_cycles_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint64)]
+    lib.grouter_gemm_cycles_read.restype = ctypes.c_int
     lib.grouter_wgrad_chunk_rows.argtypes = [vp]
     lib.grouter_wgrad_chunk_rows.restype = ctypes.c_int32
     lib.grouter_timing_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
@@ -202,6 +206,18 @@ class GrouterLayer:
     def wgrad_chunk_rows(self) -> int:
         """Rows of one expert that the weight-gradient products contract in one piece."""
         return int(self.lib.grouter_wgrad_chunk_rows(self.ctx))
+
+    def gemm_cycles_enable(self, on: bool) -> None:
+        _check(self.lib.grouter_gemm_cycles_enable(self.ctx, 1 if on else 0), "grouter_gemm_cycles_enable")
+
+    def gemm_cycles_read(self):
+        """-> {GEMM name: dict(cycles, wait_operands, wait_accumulator, tiles, k_steps)} summed over CTA pairs and launches
+        since the last read; synchronises the current stream."""
+        buf = (ctypes.c_uint64 * 30)()
+        _check(self.lib.grouter_gemm_cycles_read(self.ctx, _stream(), buf), "grouter_gemm_cycles_read")
+        names = ["gemm_up_swiglu", "gemm_down", "gemm_dH", "gemm_dX", "wgrad_down", "wgrad_gate_up"]
+        keys = ["cycles", "wait_operands", "wait_accumulator", "tiles", "k_steps"]
+        return {n: {k: int(buf[5 * i + j]) for j, k in enumerate(keys)} for i, n in enumerate(names)}
 
     def timing_read(self):
         """-> {kernel name: (total ms, launches)} since the last read; synchronises the current stream."""

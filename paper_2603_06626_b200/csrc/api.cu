@@ -175,6 +175,8 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->ev_cap = c->ev_used = 0;
   c->host_steps = 0;
   c->idle_gap_us = 0;
+  c->count_cycles = false;
+  c->d_cycles = nullptr;
   c->s_in = c->s_out = nullptr;
   for (int i = 0; i < 2; ++i) c->ev_in_fwd[i] = c->ev_in_bwd[i] = c->ev_fwd_done[i] = c->ev_bwd_done[i] = c->ev_out_done[i] = nullptr;
   {
@@ -198,6 +200,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   const size_t o_pr = take((size_t)c->max_m_tiles * 4), o_pe = take((size_t)c->max_m_tiles * 4), o_nt = take(4), o_s2p = take((size_t)c->R * 4);
   const size_t o_we = take((size_t)c->max_wchunks * 4), o_wr = take((size_t)c->max_wchunks * 4), o_wn = take((size_t)c->max_wchunks * 4), o_nw = take(4);
   const size_t o_p2s = take((size_t)c->R_pad_max * 4), o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
+  const size_t o_cy = take(6 * GEMM_CYCLE_COUNTERS * sizeof(unsigned long long));
   if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
     c->d_block = nullptr;
     grouter_destroy(c);
@@ -224,6 +227,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.ticket = reinterpret_cast<unsigned int*>(b + o_tk);
   c->pp.tile_counter = c->pp.ticket + 4;   // same 256-byte slot
   c->pp.status = reinterpret_cast<int32_t*>(b + o_st);
+  c->d_cycles = reinterpret_cast<unsigned long long*>(b + o_cy);
   *out = c;
   return GROUTER_OK;
 }
@@ -428,6 +432,22 @@ int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records) {
 int grouter_timing_gap(grouter_ctx* ctx, int32_t microseconds) {
   if (!ctx || microseconds < 0 || microseconds > 1000000) return GROUTER_ERR_INVALID_ARG;
   ctx->idle_gap_us = microseconds;
+  return GROUTER_OK;
+}
+
+int grouter_gemm_cycles_enable(grouter_ctx* ctx, int32_t on) {
+  if (!ctx) return GROUTER_ERR_INVALID_ARG;
+  ctx->count_cycles = on != 0;
+  return GROUTER_OK;
+}
+
+int grouter_gemm_cycles_read(grouter_ctx* ctx, void* stream, uint64_t* counters) {
+  if (!ctx || !counters) return GROUTER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = 6 * GEMM_CYCLE_COUNTERS * sizeof(unsigned long long);
+  if (cudaMemcpyAsync(counters, ctx->d_cycles, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaMemsetAsync(ctx->d_cycles, 0, bytes, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return GROUTER_ERR_CUDA;
   return GROUTER_OK;
 }
 

@@ -20,6 +20,7 @@ constexpr int PAIR_VALID2 = 1 << 30; // flag in PaddedPlan::pair_expert
 // the CTA pairs enough tiles when the output matrices are small.  The context picks a power of two between these bounds.
 constexpr int WGRAD_KCHUNK_MIN = 1024, WGRAD_KCHUNK_MAX = 16384;
 constexpr int WGRAD_LEN_BUCKETS = 32;   // the chunk list is ordered by chunk length in this many classes
+constexpr int GEMM_CYCLE_COUNTERS = 5;   // issuer cycles, cycles waiting for operands, for a free accumulator, tiles, k-steps
 constexpr int WCHUNK_SPLIT = 1 << 30; // flag in PaddedPlan::wchunk_expert: the expert has several chunks
 constexpr int PLAN_THREADS = 256;    // 8 warps per plan block
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
@@ -93,6 +94,8 @@ struct grouter_ctx {
   int ev_cap;
   int ev_used;
   int idle_gap_us;        // measurement aid: idle time inserted after every timed kernel (0 = none)
+  bool count_cycles;      // measurement aid: the grouped GEMMs account for their issuers' cycles
+  unsigned long long* d_cycles;   // device [6 GEMMs][GEMM_CYCLE_COUNTERS], summed over CTA pairs and launches
 };
 
 namespace grouter {

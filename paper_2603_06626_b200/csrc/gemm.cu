@@ -72,6 +72,7 @@ struct GemmParams {
   float* out_f;                // DH: dgate_part; weight gradients / DENSE: the fp32 output [E, M, N]
   int32_t* status;
   unsigned int* tile_counter;  // device scalar, zero at launch (unused by DENSE, which has no context to keep one)
+  unsigned long long* cycles;  // null, or GEMM_CYCLE_COUNTERS counters every issuer adds its account to
 };
 
 struct Tile {     // one CTA's share of a pair tile
@@ -395,17 +396,29 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       constexpr uint16_t both = 3;
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
+      // optional account of where this issuer's cycles go (measurement aid)
+      const bool count = p.cycles != nullptr;
+      long long c_acc = 0, c_full = 0, n_tiles_done = 0, n_ksteps = 0;
+      const long long c_begin = count ? clock64() : 0;
       for (int t = DYN ? next_tile() : pair_id; t < n_tiles && !*abort_flag; t = DYN ? next_tile() : t + n_pairs) {
         const Tile ti = decode_tile<MODE>(p, t, 0);
+        const long long c_t0 = count ? clock64() : 0;
         if (!ptx::mbar_wait_bounded(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) break;
+        if (count) {
+          c_acc += clock64() - c_t0;
+          n_tiles_done += 1;
+          n_ksteps += ti.steps;
+        }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
         bool ok = true;
         for (int ks = 0; ks < ti.steps; ++ks) {
+          const long long c_k0 = count ? clock64() : 0;
           if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag)) {
             ok = false;
             break;
           }
+          if (count) c_full += clock64() - c_k0;
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + s * STAGE_BYTES;
           const uint32_t sb = sa + A_BYTES;
@@ -427,6 +440,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           acc = 0;
           acc_ph ^= 1u;
         }
+      }
+      if (count) {
+        atomicAdd(p.cycles + 0, (unsigned long long)(clock64() - c_begin));
+        atomicAdd(p.cycles + 1, (unsigned long long)c_full);
+        atomicAdd(p.cycles + 2, (unsigned long long)c_acc);
+        atomicAdd(p.cycles + 3, (unsigned long long)n_tiles_done);
+        atomicAdd(p.cycles + 4, (unsigned long long)n_ksteps);
       }
     }
     __syncwarp();
@@ -756,6 +776,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.gate_is_f32 = dm.gate_dtype == GROUTER_GATE_F32;
   p.status = ctx->pp.status;
   p.tile_counter = ctx->pp.tile_counter;
+  p.cycles = ctx->count_cycles ? ctx->d_cycles + (int)mode * GEMM_CYCLE_COUNTERS : nullptr;
   Maps m;
   bool ok = true;
   const int grid = ctx->num_sms & ~1;   // whole CTA pairs, one CTA per SM

@@ -283,3 +283,46 @@ def test_whole_step_replays_from_a_cuda_graph():
     for g, x in zip(got[3:], want[3:]):      # experts cut into several chunks are summed with atomics
         assert (g - x).double().norm() <= 1e-6 * x.double().norm()
     layer.close()
+
+
+def test_issuer_cycle_accounting_counts_every_tile_and_k_step():
+    """The optional account of the MMA issuers: tile and k-step counts follow from the plan, the waits are part of the
+    total, nothing is counted while it is off, and the results do not change."""
+    from paper_2603_06626_b200 import binding
+    w = synth.WORKLOADS["small"]
+    li = synth.make_layer_inputs(w)
+    idx, gates, X, dY = to_dev(li.idx), bits_to_bf16(li.gates), bits_to_bf16(li.X), bits_to_bf16(li.dY)
+    W_gu, W_d = bits_to_bf16(li.W_gu), bits_to_bf16(li.W_d)
+    layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt)
+
+    def step():
+        layer.plan(idx)
+        Y = layer.forward(X, gates, W_gu, W_d)
+        dX = layer.backward(dY, X, gates, W_gu, W_d)[0]
+        return Y.clone(), dX.clone()
+
+    Y0, dX0 = step()
+    assert all(v == 0 for c in layer.gemm_cycles_read().values() for v in c.values())     # off by default
+    layer.gemm_cycles_enable(True)
+    Y1, dX1 = step()
+    got = layer.gemm_cycles_read()
+    layer.gemm_cycles_enable(False)
+    step()
+    assert all(v == 0 for c in layer.gemm_cycles_read().values() for v in c.values())
+    layer.check_status()
+    assert torch.equal(Y0, Y1) and torch.equal(dX0, dX1)
+
+    counts = layer.counts.cpu().numpy().astype(np.int64)
+    pair_tiles = int((((counts + 127) // 128 + 1) // 2).sum())
+    cdiv = lambda a, b: (a + b - 1) // b
+    d, F = w.d, w.ffn
+    want = {"gemm_up_swiglu": (pair_tiles * cdiv(F, 128), cdiv(d, 64)), "gemm_down": (pair_tiles * cdiv(d, 256), cdiv(F, 64)),
+            "gemm_dH": (pair_tiles * cdiv(F, 256), cdiv(d, 64)), "gemm_dX": (pair_tiles * cdiv(d, 256), cdiv(2 * F, 64))}
+    for name, (tiles, k_per_tile) in want.items():
+        c = got[name]
+        assert c["tiles"] == tiles and c["k_steps"] == tiles * k_per_tile, (name, c)
+        assert c["cycles"] >= c["wait_operands"] + c["wait_accumulator"] > 0, (name, c)
+        assert c["cycles"] >= 512 * c["k_steps"] / 74, (name, c)      # summed over the pairs: at least the tensor-core time
+    for name in ("wgrad_down", "wgrad_gate_up"):
+        assert got[name]["tiles"] > 0 and got[name]["k_steps"] >= got[name]["tiles"]
+    layer.close()
