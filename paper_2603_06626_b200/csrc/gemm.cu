@@ -202,7 +202,7 @@ __device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
   }
 }
 
-template <int MODE, bool A_MN, bool B_MN>
+template <int MODE, bool A_MN, bool B_MN, bool COUNT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
@@ -394,10 +394,17 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       constexpr uint32_t a_lbo = A_MN ? ATOM_BYTES : 16, a_sbo = 1024, a_kadv = A_MN ? 2048 : 32;
       constexpr uint32_t b_lbo = B_MN ? ATOM_BYTES : 16, b_sbo = 1024, b_kadv = B_MN ? 2048 : 32;
       constexpr uint16_t both = 3;
+      // The operand descriptors are not rebuilt per MMA: only their address field (bits 0-13, address >> 4) changes, by
+      // constants, and no carry can leave it (shared-memory addresses stay below 2^18).
+      const uint64_t da0 = ptx::make_smem_desc_sw128(smem_base, a_lbo, a_sbo);
+      const uint64_t db0 = ptx::make_smem_desc_sw128(smem_base + A_BYTES, b_lbo, b_sbo);
+      const uint32_t a_hi = (uint32_t)(da0 >> 32), b_hi = (uint32_t)(db0 >> 32);
+      uint32_t a_lo = (uint32_t)da0, b_lo = (uint32_t)db0;    // of the current stage
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
-      // optional account of where this issuer's cycles go (measurement aid)
-      const bool count = p.cycles != nullptr;
+      // account of where this issuer's cycles go (measurement aid; an instantiation of its own, because clock reads in
+      // this thread, two per k-step, cost 3-5 % of the kernel even when their results are not used)
+      constexpr bool count = COUNT;
       long long c_acc = 0, c_full = 0, n_tiles_done = 0, n_ksteps = 0;
       const long long c_begin = count ? clock64() : 0;
       for (int t = DYN ? next_tile() : pair_id; t < n_tiles && !*abort_flag; t = DYN ? next_tile() : t + n_pairs) {
@@ -420,18 +427,17 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           if (count) c_full += clock64() - c_k0;
           ptx::tc_fence_after();
-          const uint32_t sa = smem_base + s * STAGE_BYTES;
-          const uint32_t sb = sa + A_BYTES;
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            const uint64_t da = ptx::make_smem_desc_sw128(sa + kk * a_kadv, a_lbo, a_sbo);
-            const uint64_t db = ptx::make_smem_desc_sw128(sb + kk * b_kadv, b_lbo, b_sbo);
-            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (ks | kk) != 0 ? 1u : 0u);
-          }
+          for (int kk = 0; kk < BK / 16; ++kk)
+            ptx::umma_bf16_pair_split(d_tmem, a_lo + kk * (a_kadv >> 4), a_hi, b_lo + kk * (b_kadv >> 4), b_hi, idesc, (ks | kk) != 0 ? 1u : 0u);
           ptx::umma_commit_pair(empty_bar(s), both);  // stage reusable in both CTAs once these MMAs have read it
+          a_lo += STAGE_BYTES >> 4;
+          b_lo += STAGE_BYTES >> 4;
           if (++s == STAGES) {
             s = 0;
             ph ^= 1u;
+            a_lo = (uint32_t)da0;
+            b_lo = (uint32_t)db0;
           }
         }
         if (!ok) break;
@@ -735,11 +741,11 @@ struct Maps {
   CUtensorMap A, B, C0, C1, C2;
 };
 
-template <int MODE, bool A_MN, bool B_MN>
-static cudaError_t launch_t(const Maps& m, const GemmParams& p, int grid, cudaStream_t st) {
+template <int MODE, bool A_MN, bool B_MN, bool COUNT>
+static cudaError_t launch_tc(const Maps& m, const GemmParams& p, int grid, cudaStream_t st) {
   // the opt-in to more than 48 KB of dynamic shared memory is a per-device setting: once per device and instantiation
   static bool configured[64] = {};
-  auto kern = grouped_gemm_kernel<MODE, A_MN, B_MN>;
+  auto kern = grouped_gemm_kernel<MODE, A_MN, B_MN, COUNT>;
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= 64 || !configured[dev]) {
@@ -749,6 +755,14 @@ static cudaError_t launch_t(const Maps& m, const GemmParams& p, int grid, cudaSt
   }
   kern<<<grid, GEMM_THREADS, GEMM_SMEM, st>>>(m.A, m.B, m.C0, m.C1, m.C2, p);
   return cudaGetLastError();
+}
+
+template <int MODE, bool A_MN, bool B_MN>
+static cudaError_t launch_t(const Maps& m, const GemmParams& p, int grid, cudaStream_t st) {
+  if constexpr (MODE != MODE_DENSE) {
+    if (p.cycles != nullptr) return launch_tc<MODE, A_MN, B_MN, true>(m, p, grid, st);
+  }
+  return launch_tc<MODE, A_MN, B_MN, false>(m, p, grid, st);
 }
 
 static inline int cdiv(int a, int b) { return (a + b - 1) / b; }

@@ -165,14 +165,19 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 // D[tmem] (+)= A[smem] * B[smem], bf16 x bf16 -> f32, issued by one thread of the pair's leader CTA.  M = 256:
 // each CTA holds 128 rows of A and of D; B's N columns are split in halves between the two CTAs' shared memory.
 // The descriptors name shared-memory offsets that are the same in both CTAs.
-__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+// Each 64-bit descriptor is given as its two halves (the high half never changes within a kernel).
+__device__ __forceinline__ void umma_bf16_pair_split(uint32_t tmem_d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                     uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n"
       ".reg .pred p;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      ".reg .b64 da, db;\n"
+      "mov.b64 da, {%1, %2};\n"
+      "mov.b64 db, {%3, %4};\n"
+      "setp.ne.b32 p, %6, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n"
       "}\n" ::"r"(tmem_d),
-      "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // Once every tcgen05 op issued so far by this thread has completed, one arrival is delivered to the barrier at
