@@ -33,7 +33,9 @@ the only non-elementwise primitive used.
 
 Parity pins: every function in this file is pinned by tests/test_oracle_*.py
 (library stable argsort, O(R^2) brute-force ranks, hand-worked example, dense
-SwiGLU special case, torch autograd, finite differences, adjoint identity).
+SwiGLU special case, torch autograd, finite differences, adjoint identity, a
+slot-by-slot scalar-loop restatement on tiny inputs; the two error measures
+rel_frobenius and rel_rows by hand-worked numbers).
 """
 from __future__ import annotations
 
@@ -237,3 +239,23 @@ def rel_frobenius(a: np.ndarray, ref: np.ndarray) -> float:
     if den == 0.0:
         return 0.0 if num == 0.0 else float("inf")
     return float(num / den)
+
+
+def rel_rows(a: np.ndarray, ref: np.ndarray) -> np.ndarray:
+    """Per-row error of a 2-D comparison: e_i = ||a_i - ref_i||_2 / max(||ref_i||_2, rho), where rho is the root mean
+    square of the rows' norms ||ref_j||_2.  The floor rho keeps a row that is small by cancellation from dividing by
+    almost nothing; a row of an all-zero reference must match exactly (0 if it does, inf if not)."""
+    a = np.asarray(a, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    a = a.reshape(a.shape[0], -1)
+    ref = ref.reshape(ref.shape[0], -1)
+    num = np.sqrt(((a - ref) ** 2).sum(axis=1))
+    norms = np.sqrt((ref ** 2).sum(axis=1))
+    rho = np.sqrt((norms ** 2).mean()) if norms.size else 0.0
+    den = np.maximum(norms, rho)
+    out = np.zeros_like(num)
+    nz = den > 0.0
+    out[nz] = num[nz] / den[nz]
+    out[~nz & (num > 0.0)] = np.inf
+    return out
+

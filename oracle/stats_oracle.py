@@ -117,13 +117,6 @@ def local_tokens(idx: np.ndarray, node_of_expert: np.ndarray, n_nodes: int, seq_
 
 
 def place_samples(comm: np.ndarray) -> np.ndarray:
-    """best_node [S] of Algorithm 1: the node with the most local tokens, the lowest-numbered one among equals."""
-    S, N = comm.shape
-    best = np.zeros(S, dtype=np.int32)
-    for s in range(S):
-        best_node, max_comm = 0, -1
-        for n in range(N):
-            if comm[s, n] > max_comm:
-                max_comm, best_node = comm[s, n], n
-        best[s] = best_node
-    return best
+    """best_node [S]: for every sample the node holding most of its local tokens, argmax_n |T_s(n)| (Algorithm 1);
+    among nodes with equal counts the lowest-numbered one (np.argmax returns the first maximum)."""
+    return np.asarray(comm).argmax(axis=1).astype(np.int32)

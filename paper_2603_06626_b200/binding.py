@@ -291,12 +291,15 @@ def fold_greedy(coact, E_tgt: int):
     return fold
 
 
-def plan_noalloc(idx: torch.Tensor, fold_map: Optional[torch.Tensor], E_src: int, E_tgt: int, out=None, status=None):
+def plan_noalloc(idx: torch.Tensor, fold_map: Optional[torch.Tensor], E_src: int, E_tgt: int, out=None, status=None,
+                 null_status: bool = False):
     """Routing plan without a context and without any device allocation inside the library (grouter_plan_noalloc).
 
     For hosts that may not allocate: pass `out` = (counts[E_tgt], offsets[E_tgt+1], row_to_slot[R], slot_to_row[R])
     int32 device tensors and an int32[1] `status` tensor you already own, and nothing is allocated anywhere.
     When they are omitted this wrapper creates them with torch for convenience (the library still allocates nothing).
+    With `null_status` the library is given no status word at all (it then keeps the bits in its own scratch and the
+    caller learns nothing about bad ids); the last element of the result is None.
     Limits: T*k <= 524288, E_tgt <= 256.  Calls share one scratch array per GPU: keep them ordered on one stream.
     Returns (counts, offsets, row_to_slot, slot_to_row, status)."""
     lib = load_library()
@@ -305,7 +308,7 @@ def plan_noalloc(idx: torch.Tensor, fold_map: Optional[torch.Tensor], E_src: int
     i32 = dict(dtype=torch.int32, device=idx.device)
     if out is None:
         out = (torch.empty(E_tgt, **i32), torch.empty(E_tgt + 1, **i32), torch.empty(T * k, **i32), torch.empty(T * k, **i32))
-    if status is None:
+    if status is None and not null_status:
         status = torch.empty(1, **i32)
     with torch.cuda.device(idx.device):
         _check(lib.grouter_plan_noalloc(_ptr(idx), dt, _ptr(fold_map), T, k, E_src, E_tgt, _ptr(out[0]), _ptr(out[1]), _ptr(out[2]),

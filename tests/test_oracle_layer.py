@@ -212,3 +212,103 @@ def test_synth_bf16_roundtrip_and_rne():
                                   np.array([1.0, 1.0, 1.015625, -2.5, 0.0, 3.140625], dtype=np.float32))
     t = torch.tensor(a).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     np.testing.assert_array_equal(bits, t)
+
+
+def test_rel_frobenius_hand_worked():
+    """The error measure every float parity test goes through, against numbers worked by hand."""
+    assert orc.rel_frobenius([3.0, 4.0], [0.0, 0.0]) == float("inf")            # zero reference, non-zero input
+    assert orc.rel_frobenius([0.0, 0.0], [0.0, 0.0]) == 0.0                     # zero against zero
+    assert orc.rel_frobenius([1.0, 2.0, 2.0], [1.0, 2.0, 2.0]) == 0.0
+    # a - ref = [0, 0, 2]: ||.|| = 2; ||ref|| = sqrt(1 + 4 + 0) = sqrt(5)
+    assert orc.rel_frobenius([1.0, 2.0, 2.0], [1.0, 2.0, 0.0]) == pytest.approx(2.0 / 5.0 ** 0.5, rel=1e-15)
+    # not symmetric: the reference is the denominator.  a - ref = [0, 0, -2]; ||ref|| = 3
+    assert orc.rel_frobenius([1.0, 2.0, 0.0], [1.0, 2.0, 2.0]) == pytest.approx(2.0 / 3.0, rel=1e-15)
+    # 2-D: differences 1, 0, 0, 2 -> sqrt(5); reference entries 1, 2, 3, 4 -> sqrt(30)
+    assert orc.rel_frobenius([[2.0, 2.0], [3.0, 6.0]], [[1.0, 2.0], [3.0, 4.0]]) == pytest.approx((5.0 / 30.0) ** 0.5, rel=1e-15)
+    # scale-free in the pair, first order in a uniform relative error
+    ref = np.arange(1.0, 7.0).reshape(2, 3)
+    assert orc.rel_frobenius(1.001 * ref, ref) == pytest.approx(1e-3, rel=1e-9)
+    assert orc.rel_frobenius(7.0 * 1.001 * ref, 7.0 * ref) == pytest.approx(1e-3, rel=1e-9)
+    # float32 input is widened, not the reference narrowed
+    assert orc.rel_frobenius(np.array([1.0, 1.0], dtype=np.float32), np.array([1.0, 1.0 + 2.0 ** -40])) > 0.0
+
+
+def test_rel_rows_hand_worked():
+    ref = np.array([[3.0, 4.0], [0.0, 0.0], [6.0, 8.0]])          # row norms 5, 0, 10; rms = sqrt((25 + 0 + 100) / 3) = 6.4549...
+    a = np.array([[3.0, 5.0], [0.3, 0.4], [6.0, 8.0]])            # row errors 1, 0.5, 0
+    rho = (125.0 / 3.0) ** 0.5
+    np.testing.assert_allclose(orc.rel_rows(a, ref), [1.0 / rho, 0.5 / rho, 0.0], rtol=1e-15)
+    # a row above the floor is divided by its own norm: error 1 on the row of norm 10
+    a2 = ref.copy(); a2[2, 0] += 1.0
+    np.testing.assert_allclose(orc.rel_rows(a2, ref), [0.0, 0.0, 0.1], rtol=1e-15)
+    # all-zero reference: exact match or inf
+    z = np.zeros((2, 3))
+    assert orc.rel_rows(z, z).tolist() == [0.0, 0.0]
+    assert orc.rel_rows(np.array([[0.0, 0.0, 0.0], [0.0, 1e-30, 0.0]]), z).tolist() == [0.0, float("inf")]
+    # trailing axes are flattened into the row: [2, 2, 2] is two rows of four
+    r3 = np.arange(8.0).reshape(2, 2, 2)
+    a3 = r3.copy(); a3[1, 1, 1] += 2.0                            # row norms sqrt(14), sqrt(126); rms = sqrt(70)
+    np.testing.assert_allclose(orc.rel_rows(a3, r3), [0.0, 2.0 / 126.0 ** 0.5], rtol=1e-15)
+    # one wrong row in a thousand stands out by orders of magnitude where the Frobenius ratio hardly moves
+    rng = np.random.default_rng(0)
+    big = rng.standard_normal((1000, 64))
+    bad = big * (1.0 + 3e-3 * rng.standard_normal(big.shape))
+    bad[417] = rng.standard_normal(64)
+    assert orc.rel_frobenius(bad, big) < 5e-2 and orc.rel_rows(bad, big)[417] > 1.0
+    assert np.delete(orc.rel_rows(bad, big), 417).max() < 1e-2
+
+
+def _scalar_loop_layer(X, dY, W_gu, W_d, idx, gates, fm, E_tgt):
+    """Eq. 1 and its gradients slot by slot with scalar loops only (no matmul, no masks, no grouping by expert):
+    for every slot (t, j): e = m[idx], a = W_g x, u = W_u x, h = silu(a) u, o = W_d h, y_t += g o, and the chain rule
+    written out element by element."""
+    import math
+    T, d = X.shape
+    k = idx.shape[1]
+    F = W_gu.shape[1] // 2
+    Y = np.zeros((T, d)); dX = np.zeros((T, d)); dg = np.zeros((T, k))
+    dWgu = np.zeros((E_tgt, 2 * F, d)); dWd = np.zeros((E_tgt, d, F))
+    for t in range(T):
+        for j in range(k):
+            e = int(idx[t, j]) if fm is None else int(fm[int(idx[t, j])])
+            g = gates[t, j]
+            a = [sum(W_gu[e, f, c] * X[t, c] for c in range(d)) for f in range(F)]
+            u = [sum(W_gu[e, F + f, c] * X[t, c] for c in range(d)) for f in range(F)]
+            sg = [1.0 / (1.0 + math.exp(-a[f])) for f in range(F)]
+            h = [a[f] * sg[f] * u[f] for f in range(F)]
+            o = [sum(W_d[e, c, f] * h[f] for f in range(F)) for c in range(d)]
+            for c in range(d):
+                Y[t, c] += g * o[c]
+            dg[t, j] = sum(dY[t, c] * o[c] for c in range(d))
+            dh = [sum(g * dY[t, c] * W_d[e, c, f] for c in range(d)) for f in range(F)]
+            for c in range(d):
+                for f in range(F):
+                    dWd[e, c, f] += g * dY[t, c] * h[f]
+            for f in range(F):
+                da = dh[f] * u[f] * sg[f] * (1.0 + a[f] * (1.0 - sg[f]))
+                du = dh[f] * a[f] * sg[f]
+                for c in range(d):
+                    dWgu[e, f, c] += da * X[t, c]
+                    dWgu[e, F + f, c] += du * X[t, c]
+                    dX[t, c] += W_gu[e, f, c] * da + W_gu[e, F + f, c] * du
+    return Y, dX, dg, dWgu, dWd
+
+
+@pytest.mark.parametrize("fold_to,distinct", [(None, True), (2, True), (None, False)])
+def test_against_scalar_loops(fold_to, distinct):
+    """The oracle groups slots by expert and multiplies matrices with a library routine; the same quantities from
+    scalar loops over single slots (no library contraction anywhere) must agree to rounding."""
+    T, d, F, E, k = 7, 5, 3, 4, 2
+    X, dY, W_gu, W_d, idx, gates, fm = _rand_layer(12, T, d, F, E, k, fold_to, distinct)
+    E_tgt = fold_to or E
+    Wt = orc.Weights(W_gu, W_d)
+    Y = orc.moe_forward(X, idx, gates, Wt, E_tgt, fm)
+    dX, dg, dW = orc.moe_backward(dY, X, idx, gates, Wt, E_tgt, fm)
+    sY, sdX, sdg, sdWgu, sdWd = _scalar_loop_layer(X, dY, W_gu, W_d, idx, gates, fm, E_tgt)
+    np.testing.assert_allclose(Y, sY, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dX, sdX, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(dg, sdg, rtol=1e-12, atol=1e-12)
+    for e in range(E_tgt):
+        np.testing.assert_allclose(dW[e][0], sdWgu[e], rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(dW[e][1], sdWd[e], rtol=1e-12, atol=1e-12)
+

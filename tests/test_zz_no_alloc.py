@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import grouter_oracle as orc
 from paper_2603_06626_b200 import synth
 from tests.gpu_util import to_dev
 
@@ -55,10 +56,12 @@ def test_noalloc_plan_matches_context_plan_twice_in_a_row():
         fm = None if fm_np is None else to_dev(fm_np)
         results.append(binding.plan_noalloc(to_dev(idx_np), fm, E_src, E_tgt, out=out, status=status))
     torch.cuda.synchronize()
-    for got, want in zip(results, expected):
+    for got, want, (idx_np, fm_np, _, E_tgt) in zip(results, expected, cases):
         assert int(got[4].item()) == 0
         for g, w, name in zip(got[:4], want, NAMES):
             assert torch.equal(g, w), name
+        for g, o, name in zip(got[:4], orc.plan(idx_np, fm_np, E_tgt), NAMES):      # and against the CPU oracle directly
+            assert np.array_equal(g.cpu().numpy(), o), name
 
     # a bad id is reported through the caller's status word, nothing faults, every slot is still counted
     bad = np.zeros((100, 2), dtype=np.uint8)
@@ -72,6 +75,37 @@ def test_noalloc_plan_matches_context_plan_twice_in_a_row():
     assert int(got[4].item()) == 0
     for g, w, name in zip(got[:4], expected[1], NAMES):
         assert torch.equal(g, w), name
+
+
+def test_noalloc_plan_at_the_limits_of_its_scratch_allocates_nothing():
+    """The largest problem the fixed scratch is laid out for: T*k = 524288 slots over 256 experts, almost all of which
+    get one or two rows (so the padded layout is at its longest), 32-bit ids, and no status word from the caller.
+    Device memory in use must be the same before and after the call."""
+    from paper_2603_06626_b200 import binding
+    T, k, E = 65536, 8, 256
+    rng = np.random.default_rng(5)
+    idx_np = rng.integers(0, 2, size=(T, k)).astype(np.int32)           # two heavy experts ...
+    light = rng.choice(T * k, size=380, replace=False)
+    idx_np.reshape(-1)[light] = rng.integers(2, E, size=380)            # ... and 254 that get a row or two
+    want = orc.plan(idx_np, None, E)
+    assert (want[0][2:] <= 8).all() and (want[0] > 0).sum() > 150
+    idx = to_dev(idx_np)
+    i32 = dict(dtype=torch.int32, device="cuda:0")
+    out = (torch.empty(E, **i32), torch.empty(E + 1, **i32), torch.empty(T * k, **i32), torch.empty(T * k, **i32))
+    binding.plan_noalloc(idx, None, E, E, out=out, null_status=True)      # first call on the device: looks the scratch address up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for o in out:
+        o.fill_(-7)
+    got = binding.plan_noalloc(idx, None, E, E, out=out, null_status=True)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and got[4] is None
+    for g, o, name in zip(got[:4], want, NAMES):
+        assert np.array_equal(g.cpu().numpy(), o), name
+    ctx = _with_context(idx_np, None, E, E)
+    for g, c, name in zip(got[:4], ctx, NAMES):
+        assert torch.equal(g, c), name
 
 
 def test_noalloc_plan_rejects_sizes_beyond_its_scratch():
