@@ -55,26 +55,53 @@ def kernel_source_tag() -> str:
     return h.hexdigest()[:12]
 
 
-def recorded_traffic(workload: str, kernel: str):
-    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
-    profiles/dram_traffic.txt, or None when there is no capture of this kernel on this workload with this build."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
-    if not os.path.exists(path):
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+
+
+def algorithmic_dram_bytes(w: synth.Workload, kernel: str) -> float:
+    """Bytes a launch must move through DRAM if every operand is read once and every result written once (valid
+    rows only).  Used to scale DRAM counters captured on a small workload to the benchmarked one."""
+    R, T, d, F, E = float(w.R), float(w.T), float(w.d), float(w.ffn), float(w.E_tgt)
+    act_d, act_f, w_gu, w_d = R * d * 2, R * F * 2, E * 2 * F * d * 2, E * d * F * 2
+    table = {
+        "gemm_up_swiglu": act_d + w_gu + 3 * act_f, "gemm_down": act_f + w_d + act_d,
+        "gemm_dH": act_d + w_d + 2 * act_f + 2 * act_f + 2 * ((w.ffn + 255) // 256) * R * 4, "gemm_dX": 2 * act_f + w_gu + act_d,
+        "wgrad_down": act_d + act_f + 2 * w_d, "wgrad_gate_up": 2 * act_f + act_d + 2 * w_gu,
+        "gather_X": (T + R) * d * 2, "combine_Y": (T + R) * d * 2, "gather_dY": (T + R) * d * 2, "reduce_dX": (T + R) * d * 2,
+    }
+    return table.get(kernel, 0.0)
+
+
+def recorded_traffic(w: synth.Workload, kernel: str):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of `kernel` on workload `w`.
+
+    profiles/dram_traffic.txt holds one-pass ncu counters taken on a workload of a few GB (lines: workload kernel bytes
+    source-tag).  A line for `w` itself is used as it stands; otherwise the small workload's figure is scaled by the
+    ratio of the two workloads' algorithmic bytes (DRAM traffic of these kernels follows their operand and result sizes:
+    the capture reads within a few per cent of the algorithmic bytes).  None when the CUDA sources have changed since
+    the capture (other source tag) or there is no line for the kernel."""
+    if not os.path.exists(TRAFFIC_FILE):
         return None
     tag = kernel_source_tag()
-    for line in open(path):
+    scaled = None
+    for line in open(TRAFFIC_FILE):
         parts = line.split()
-        if len(parts) >= 4 and not line.startswith("#") and parts[0] == workload and parts[1] == kernel and parts[3] == tag:
+        if len(parts) < 4 or line.startswith("#") or parts[1] != kernel or parts[3] != tag:
+            continue
+        if parts[0] == w.name:
             return float(parts[2])
-    return None
+        src = synth.WORKLOADS.get(parts[0])
+        if src is not None and algorithmic_dram_bytes(src, kernel) > 0:
+            scaled = float(parts[2]) * algorithmic_dram_bytes(w, kernel) / algorithmic_dram_bytes(src, kernel)
+    return scaled
 
 
-def plan_at_scale(dev, T=1 << 22, k=8, E=128, iters=5):
-    """The plan build at a size where bytes, not launch latency, decide its time: uniform ids, T*k = 2^25 slots.
-    Algorithmic bytes: ids read twice (histogram pass, permutation pass) and the two permutations written."""
+def plan_at_scale(dev, T=1 << 24, k=8, E=128, iters=5):
+    """The plan build at a size where bytes, not launch latency, decide its time: uniform 8-bit ids, T*k = 2^27 slots.
+    Algorithmic bytes: the ids read once, the two permutations written, counts and offsets written."""
     import torch
     from paper_2603_06626_b200 import binding
-    layer = binding.GrouterLayer(T, 8, 8, E, k, device=str(dev))
+    layer = binding.GrouterLayer(T, 8, 8, E, k, device=str(dev), plan_only=True)
     g = torch.Generator(device=dev)
     g.manual_seed(7)
     idx = torch.randint(0, E, (T, k), dtype=torch.uint8, device=dev, generator=g)
@@ -92,8 +119,9 @@ def plan_at_scale(dev, T=1 << 22, k=8, E=128, iters=5):
     R = T * k
     assert int(layer.counts.sum().item()) == R
     layer.close()
-    by = 2.0 * R + 2.0 * R * 4
-    return {"T": T, "k": k, "E": E, "ms": ms, "algorithmic_bytes": by, "gbs": by / (ms * 1e-3) / 1e9}
+    by = 1.0 * R + 2.0 * R * 4 + (2 * E + 1) * 4
+    return {"T": T, "k": k, "E": E, "ms": ms, "algorithmic_bytes": by, "gbs": by / (ms * 1e-3) / 1e9,
+            "note": "bytes as defined for the plan: ids read once; the two kernels that read the ids move 1 byte per slot more"}
 
 
 def router_head_leg(dev, T=32768, d_h=512, E_src=128, E_tgt=128, k=8, iters=20):
@@ -192,7 +220,7 @@ def kernel_work(w: synth.Workload, counts: np.ndarray, chunk_rows: int):
         "gemm_dX": ("flop", 2 * dF), "wgrad_gate_up": ("flop", 2 * dF),
         "gather_X": ("byte", (T + R) * d * 2.0), "combine_Y": ("byte", (T + R) * d * 2.0),
         "gather_dY": ("byte", (T + R) * d * 2.0), "reduce_dX": ("byte", (T + R) * d * 2.0),
-        "plan_hist": ("byte", R * idb + 0.0), "plan_permute": ("byte", R * idb + 2.0 * R * 4),
+        "plan_hist": ("byte", R * idb + 0.0), "plan_permute": ("byte", R * idb + 2.0 * R * 4), "plan_scan": ("byte", (2.0 * w.E_tgt + 1) * 4),
         "zero_split_dW": ("byte", n_split * 3.0 * d * F * 4),
     }
 
@@ -249,37 +277,54 @@ class ClockSampler:
         return out
 
 
-def oracle_sample_tokens_per_sec(w: synth.Workload, li, n_tokens: int):
-    """The fp64 oracle, as it stands, on the first n_tokens tokens of the workload (full fwd + bwd incl. every
-    expert's weight gradients for those tokens).  Returns (tokens/s, seconds, threads)."""
-    from oracle import grouter_oracle as orc
+def blas_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
-        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
     except Exception:
-        threads = os.cpu_count() or 1
-    sub = slice(0, n_tokens)
-    X = synth.bf16_bits_to_f64(li.X[sub]); dY = synth.bf16_bits_to_f64(li.dY[sub]); gates = synth.bf16_bits_to_f64(li.gates[sub])
-    idx = li.idx[sub]
-    if li.W_gu is not None:
-        getter = lambda e: (synth.bf16_bits_to_f64(li.W_gu[e]), synth.bf16_bits_to_f64(li.W_d[e]))  # noqa: E731
-    else:
-        cache = {}
+        return os.cpu_count() or 1
 
-        def getter(e):
-            if e not in cache:
-                cache[e] = (synth.expert_W_gu(w, e), synth.expert_W_d(w, e))
-            return synth.bf16_bits_to_f64(cache[e][0]), synth.bf16_bits_to_f64(cache[e][1])
-        used = np.unique(orc.fold_ids(idx, li.fold_map))
-        for e in used:           # draw the weights before the clock starts
-            getter(int(e))
-    weights = orc.Weights(getter=getter, ffn=w.ffn)
-    used = [int(e) for e in np.unique(orc.fold_ids(idx, li.fold_map))]
-    t0 = time.perf_counter()
-    orc.moe_forward(X, idx, gates, weights, w.E_tgt, li.fold_map)
-    orc.moe_backward(dY, X, idx, gates, weights, w.E_tgt, li.fold_map, experts=used)
-    dt = time.perf_counter() - t0
-    return n_tokens / dt, dt, threads
+
+def oracle_sample_tokens_per_sec(w: synth.Workload, li, n_experts: int = 1):
+    """The fp64 oracle, as it stands, on whole experts: forward and full backward (dX, dgates, and the expert's dW_gu,
+    dW_d) of the tokens routed to the `n_experts` experts whose loads are closest to the median load, each expert's
+    weights widened to fp64 before the clock starts.  The layer costs the same arithmetic per routed row whichever
+    expert owns it, so tokens/s of the whole workload = (T * k / rows timed) ... / seconds, i.e. the timed rows
+    extrapolated to all T * k routed rows.  Returns (tokens/s extrapolated, seconds, BLAS threads, description)."""
+    from oracle import grouter_oracle as orc
+    ids = orc.fold_ids(li.idx, li.fold_map).reshape(w.T, w.k)
+    loads = np.bincount(ids.reshape(-1), minlength=w.E_tgt)
+    nz = np.nonzero(loads)[0]
+    order = nz[np.argsort(np.abs(loads[nz] - np.median(loads[nz])), kind="stable")]
+    chosen = [int(e) for e in order[:n_experts]]
+    cache = {}
+    for e in chosen:                      # weights drawn and widened before the clock starts
+        if li.W_gu is not None:
+            cache[e] = (synth.bf16_bits_to_f64(li.W_gu[e]), synth.bf16_bits_to_f64(li.W_d[e]))
+        else:
+            cache[e] = (synth.bf16_bits_to_f64(synth.expert_W_gu(w, e)), synth.bf16_bits_to_f64(synth.expert_W_d(w, e)))
+    weights = orc.Weights(getter=lambda e: cache[e], ffn=w.ffn)
+    pairs_all = int(np.unique(np.arange(w.T, dtype=np.int64)[:, None] * w.E_tgt + ids).shape[0])    # (token, expert) evaluations of f_e
+    pairs = 0
+    dt = 0.0
+    for e in chosen:
+        hit = ids == e
+        tok = np.nonzero(hit.any(axis=1))[0]
+        # sub-problem: these tokens, one slot each on expert e carrying the token's coefficient r(x)_e (Eq. 1)
+        idx_e = np.full((tok.shape[0], 1), e, dtype=np.int64)
+        gates_e = np.where(hit[tok], synth.bf16_bits_to_f64(li.gates[tok]), 0.0).sum(axis=1, keepdims=True)
+        X = synth.bf16_bits_to_f64(li.X[tok])
+        dY = synth.bf16_bits_to_f64(li.dY[tok])
+        t0 = time.perf_counter()
+        orc.moe_forward(X, idx_e, gates_e, weights, w.E_tgt)
+        orc.moe_backward(dY, X, idx_e, gates_e, weights, w.E_tgt, experts=[e])
+        dt += time.perf_counter() - t0
+        pairs += int(tok.shape[0])
+    tokens_per_s = w.T / (dt * pairs_all / pairs)
+    what = (f"fp64 numpy oracle on whole experts: the {len(chosen)} expert(s) of median load ({pairs} of the workload's {pairs_all} "
+            f"(token, expert) evaluations), forward + full backward incl. the expert's weight gradients, weights widened outside "
+            f"the clock; extrapolated to the whole workload (same arithmetic per evaluation)")
+    return tokens_per_s, dt, blas_threads(), what
 
 
 def run_reference(args):
@@ -289,16 +334,17 @@ def run_reference(args):
         return
     w = synth.WORKLOADS[args.workload]
     li = synth.make_layer_inputs(w, with_weights=False)
-    n = args.ref_tokens
     times = []
     threads = 1
+    value = 0.0
+    sample = ""
     for i in range(args.warmup + args.steps):
-        _, dt, threads = oracle_sample_tokens_per_sec(w, li, n)
+        v, dt, threads, sample = oracle_sample_tokens_per_sec(w, li, 1)
         if i >= args.warmup:
-            times.append(dt)
-    total = sum(times)
-    value = n * len(times) / total
-    sample = f"first {n} tokens of the workload per step (all their experts, fwd + full bwd), fp64 numpy"
+            times.append((v, dt))
+    total = sum(dt for _, dt in times)
+    value = sum(v * dt for v, dt in times) / total            # time-weighted: total tokens' worth of work / total seconds
+    sample = "per step: " + sample
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times), "higher_is_better": True, "scaling": "weak",
@@ -325,13 +371,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="large", choices=list(synth.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--ref-tokens", type=int, default=2, help="tokens per step of the reference arm's oracle sample")
-    ap.add_argument("--cpu-baseline-tokens", type=int, default=48)
+    ap.add_argument("--cpu-baseline-experts", type=int, default=12, help="whole experts the CPU baseline times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-plan-scale", action="store_true")
     ap.add_argument("--no-isolated", action="store_true")
-    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=0, help="steps of the end-to-end leg (0: as many as --steps)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
@@ -387,7 +432,7 @@ def main():
     layer.check_status()
     barrier()
     torch.cuda.synchronize()
-    layer.timing_enable(len(binding.KERNEL_SLOTS) * args.steps)
+    # ---- the headline: K whole steps back to back, nothing but the step's own launches on the stream ----
     wall0 = time.time()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps - 1)]   # between steps: median / best step
@@ -404,12 +449,27 @@ def main():
     barrier()
     ms_total = ev0.elapsed_time(ev1)
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
-    per_kernel = layer.timing_read()
-    layer.timing_enable(0)
     layer.check_status()
     ms_total = shard.max_over_ranks(ms_total, dev, world)
     ms_step = ms_total / args.steps
     value = shard.job_tokens_per_sec(world, w.T, ms_step)
+
+    # ---- the per-kernel table: a pass of its own with an event pair around every launch (not part of `value`) ----
+    n_table = min(args.steps, 10)
+    layer.timing_enable(len(binding.KERNEL_SLOTS) * n_table)
+    for _ in range(n_table):
+        step()
+    per_kernel = layer.timing_read()
+    layer.timing_enable(0)
+    layer.check_status()
+    # the plan build alone, back to back on the stream (its three launches are too short for event pairs around each)
+    pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pe0.record()
+    for _ in range(50):
+        layer.plan(idx, fm)
+    pe1.record()
+    torch.cuda.synchronize()
+    plan_alone_ms = pe0.elapsed_time(pe1) / 50
 
     # ---- every kernel alone: 30 ms of idle time after each launch, so that none starts at the power cap ----
     isolated = None
@@ -444,6 +504,8 @@ def main():
 
     # ---- end to end: host buffers in, host results out, every step ----
     e2e = None
+    if args.e2e_steps <= 0:
+        args.e2e_steps = args.steps
     if not args.no_e2e:
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()  # noqa: E731
         # two sets of pinned host buffers, used alternately: one step stays in flight while the host reads the previous one
@@ -517,9 +579,9 @@ def main():
                 ent["alone_frac_of_hbm"] = ent["alone_gbs"] / peaks["hbm_gbs"]
         kernels[name] = ent
     dom = max(GEMM_SLOTS, key=lambda k: per_kernel[k][0])
-    traffic = recorded_traffic(w.name, dom)
+    traffic = recorded_traffic(w, dom)
     for name, ent in kernels.items():
-        ent["traffic"] = recorded_traffic(w.name, name)
+        ent["traffic"] = recorded_traffic(w, name)
     roofline = {"kernel": dom, "bound": "tensor", "achieved": kernels[dom]["tflops"], "peak": peaks["bf16_tflops_sustained"],
                 "unit": "TFLOP/s", "frac": kernels[dom]["tflops"] / peaks["bf16_tflops_sustained"], "traffic": traffic,
                 "peak_source": f"{peak_src} cuBLAS bf16, sustained (kernel timed inside a long step); burst peak "
@@ -535,16 +597,16 @@ def main():
     # one routing plan can serve every layer of the model, forward and backward (the router runs before the model):
     # the same step with the plan's two launches left out of the time
     n_timed = per_kernel["gemm_up_swiglu"][1]
-    plan_ms = (per_kernel["plan_hist"][0] + per_kernel["plan_permute"][0]) / max(n_timed, 1)
-    plan = {"ms": plan_ms, "share_of_step": plan_ms / ms_step,
-            "value_plan_amortised": value * ms_step / (ms_step - plan_ms) if ms_step > plan_ms else None,
+    plan_ms = (per_kernel["plan_hist"][0] + per_kernel["plan_scan"][0] + per_kernel["plan_permute"][0]) / max(n_timed, 1)
+    plan = {"ms": plan_alone_ms, "ms_event_pairs_in_step": plan_ms, "launches": 3, "share_of_step": plan_alone_ms / ms_step,
+            "value_plan_amortised": value * ms_step / (ms_step - plan_alone_ms) if ms_step > plan_alone_ms else None,
             "note": "tokens/s if the plan is built once and reused by many layers"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
         "ms_per_step": ms_step, "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_best": step_ms[0], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(base, world), "clocks": clocks,
-        "gpu_launches": int(sum(v[1] for v in per_kernel.values())), "roofline": roofline, "kernels": kernels, "gemm_summary": summary, "plan": plan,
+        "gpu_launches": int(sum(v[1] for v in per_kernel.values()) // max(n_timed, 1) * args.steps), "roofline": roofline, "kernels": kernels, "gemm_summary": summary, "plan": plan,
         "gemm_cycles": gemm_cycles,
         "load_stats": synth.load_stats(li.idx, li.fold_map, w.E_tgt),
     }
@@ -552,6 +614,8 @@ def main():
         line["e2e"] = e2e
     if world == 1 and not args.no_plan_scale:
         layer.close()
+        torch.cuda.synchronize()
+        time.sleep(3.0)     # the step loop ran at the power cap; these short kernels are timed on a GPU that has settled
         ps = plan_at_scale(dev)
         ps["frac_of_hbm"] = ps["gbs"] / peaks["hbm_gbs"]
         line["plan_scaled"] = ps
@@ -561,10 +625,9 @@ def main():
         if w.E_src <= 256 and w.T % 4096 == 0:
             line["routing_stats"] = routing_stats_leg(dev, idx, w.E_src)
     if world == 1 and not args.no_cpu_baseline:
-        v, dt, threads = oracle_sample_tokens_per_sec(w, li, args.cpu_baseline_tokens)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt,
-                                "sample": f"first {args.cpu_baseline_tokens} tokens of the workload (all their experts, fwd + full bwd), "
-                                          "fp64 numpy oracle"}
+        v, dt, threads, what = oracle_sample_tokens_per_sec(w, li, args.cpu_baseline_experts)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt, "sample": what,
+                                "extrapolated": True}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -69,8 +69,9 @@ typedef struct {
 } grouter_dims;
 
 /* Creates a context for one layer shape on the current CUDA device.  Host call;
- * the only call that allocates: a few MB of device memory for the padded copy
- * of the plan, the tile list, per-block histograms and the status word.
+ * the only call that allocates: device memory for the padded layout, the tile
+ * and chunk lists, per-block histograms (4 * E_tgt bytes per 4096-16384 slots)
+ * and the status word.
  * Errors: INVALID_ARG, UNSUPPORTED, NO_DEVICE, CUDA. */
 int grouter_create(grouter_ctx** out, const grouter_dims* dims);
 void grouter_destroy(grouter_ctx* ctx);
@@ -98,9 +99,12 @@ size_t grouter_host_staging_bytes(const grouter_dims* dims);
  *   fold_map    [E_src] int32 in [0,E_tgt), or NULL for the identity
  *   counts      [E_tgt] int32 out          offsets     [E_tgt+1] int32 out
  *   row_to_slot [R] int32 out              slot_to_row [R] int32 out
- * The context keeps a 128-row-padded copy of the plan for fwd/bwd; one plan
- * may serve any number of fwd/bwd calls (all MoE layers of a micro-batch share
- * the same frozen router; section "Decoupled Structure Extraction").
+ * fwd and bwd read offsets, row_to_slot and slot_to_row from these arrays (the
+ * context keeps the pointers, the 128-row-padded layout and the GEMMs' work
+ * lists): leave them in place and unchanged until the last fwd/bwd that uses
+ * this plan has completed.  One plan may serve any number of fwd/bwd calls (all
+ * MoE layers of a micro-batch share the same frozen router; section "Decoupled
+ * Structure Extraction").
  * An id outside [0,E_src) or a fold target outside [0,E_tgt) is treated as
  * expert 0 and sets the sticky status GROUTER_ERR_BAD_INDEX. */
 int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
@@ -112,7 +116,7 @@ int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int
  * whole device to a pooling allocator, runs under a fixed memory budget, or
  * cannot afford the device-wide synchronisation of an allocation inside its loop
  * calls this instead: the scratch is a fixed array inside the library image
- * (about 4.6 MB, present on every GPU that loads the library until the process
+ * (about 0.3 MB, present on every GPU that loads the library until the process
  * exits), and the call makes no cudaMalloc/cudaFree and uses no allocating
  * library routine.
  *   Same definition and outputs as grouter_plan (counts, offsets, row_to_slot,
@@ -242,8 +246,8 @@ const char* grouter_strerror(int code);
  * elapsed milliseconds and launch counts per kernel slot, and empties the pool.
  * Slots: 0 plan_hist, 1 plan_permute, 2 gather_X, 3 gemm_up_swiglu, 4 gemm_down,
  * 5 combine_Y, 6 gather_dY, 7 gemm_dH, 8 wgrad_down, 9 gemm_dX, 10 wgrad_gate_up,
- * 11 reduce_dX, 12 zero_split_dW.   total_ms, launches: HOST arrays of GROUTER_NUM_KERNELS entries. */
-#define GROUTER_NUM_KERNELS 13
+ * 11 reduce_dX, 12 zero_split_dW, 13 plan_scan.   total_ms, launches: HOST arrays of GROUTER_NUM_KERNELS entries. */
+#define GROUTER_NUM_KERNELS 14
 int grouter_timing_enable(grouter_ctx* ctx, int32_t n_records);
 /* While timing is enabled, let `microseconds` (0..1000000; 0 = off, the default) of idle time pass on the stream after
  * every timed kernel, so that each kernel is measured on a GPU that is not already at its power cap: the figure to

@@ -24,7 +24,7 @@ EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grou
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
            "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
-                "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW"]
+                "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW", "plan_scan"]
 
 
 class GrouterDims(ctypes.Structure):
@@ -47,8 +47,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
         return _lib
     if path is None:
         path = _build.LIB
-        if not os.path.exists(path) or os.environ.get("GROUTER_REBUILD"):
-            _build.build()
+        _build.build(force=bool(os.environ.get("GROUTER_REBUILD")))     # returns at once when the library is newer than every source
     lib = ctypes.CDLL(path)
     vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
     lib.grouter_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(GrouterDims)]
@@ -126,7 +125,8 @@ class GrouterLayer:
     """One layer shape: owns the context and the workspace; thin calls into the C ABI."""
 
     def __init__(self, T: int, d: int, ffn: int, E_src: int, k: int, E_tgt: Optional[int] = None, idx_dtype: int = IDX_U8,
-                 gate_dtype: int = GATE_BF16, device: str = "cuda:0", host_staging: bool = False, flags: int = 0):
+                 gate_dtype: int = GATE_BF16, device: str = "cuda:0", host_staging: bool = False, flags: int = 0,
+                 plan_only: bool = False):
         self.lib = load_library()
         self.device = torch.device(device)
         self.dims = GrouterDims(T, d, ffn, E_src, E_src if E_tgt is None else E_tgt, k, idx_dtype, gate_dtype, flags)
@@ -143,7 +143,8 @@ class GrouterLayer:
             self.workspace_bytes = n
             if host_staging:
                 n += self.lib.grouter_host_staging_bytes(ctypes.byref(self.dims))
-            self.workspace = torch.empty(n, dtype=torch.uint8, device=self.device)
+            # plan_only: the caller only builds plans with this context (no forward/backward), so no workspace is needed
+            self.workspace = None if plan_only else torch.empty(n, dtype=torch.uint8, device=self.device)
         i32 = dict(dtype=torch.int32, device=self.device)
         self.counts = torch.empty(self.E_tgt, **i32)
         self.offsets = torch.empty(self.E_tgt + 1, **i32)

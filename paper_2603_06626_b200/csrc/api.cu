@@ -168,7 +168,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
     c->pp.wgrad_chunk_blocks = chunk / ROW_TILE;
     c->max_wchunks = dims->E_tgt + (int)(c->R_pad_max / chunk) + 1;
   }
-  c->geom = plan_geom(c->R);
+  c->geom = plan_geom(c->R, dims->E_src, dims->E_tgt);
   c->planned = c->forwarded = false;
   c->ev_start = c->ev_stop = nullptr;
   c->ev_slot = nullptr;
@@ -196,10 +196,10 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   const int E = dims->E_tgt;
   size_t off = 0;
   auto take = [&](size_t n) { size_t o = off; off += align_up(n, 256); return o; };
-  const size_t o_pad = take((size_t)(E + 1) * 4), o_shift = take((size_t)E * 4), o_pb = take((size_t)E * 4);
-  const size_t o_pr = take((size_t)c->max_m_tiles * 4), o_pe = take((size_t)c->max_m_tiles * 4), o_nt = take(4), o_s2p = take((size_t)c->R * 4);
+  const size_t o_pad = take((size_t)(E + 1) * 4), o_shift = take((size_t)E * 4), o_pb = take((size_t)E * 4), o_pp = take((size_t)(E + 1) * 4);
+  const size_t o_pr = take((size_t)c->max_m_tiles * 4), o_pe = take((size_t)c->max_m_tiles * 4), o_nt = take(4);
   const size_t o_we = take((size_t)c->max_wchunks * 4), o_wr = take((size_t)c->max_wchunks * 4), o_wn = take((size_t)c->max_wchunks * 4), o_nw = take(4);
-  const size_t o_p2s = take((size_t)c->R_pad_max * 4), o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
+  const size_t o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
   const size_t o_cy = take(6 * GEMM_CYCLE_COUNTERS * sizeof(unsigned long long));
   if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
     c->d_block = nullptr;
@@ -214,6 +214,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.pad_offsets = reinterpret_cast<int32_t*>(b + o_pad);
   c->pp.row_shift = reinterpret_cast<int32_t*>(b + o_shift);
   c->pp.pad_begin = reinterpret_cast<int32_t*>(b + o_pb);
+  c->pp.pair_prefix = reinterpret_cast<int32_t*>(b + o_pp);
   c->pp.pair_row0 = reinterpret_cast<int32_t*>(b + o_pr);
   c->pp.pair_expert = reinterpret_cast<int32_t*>(b + o_pe);
   c->pp.n_pair_tiles = reinterpret_cast<int32_t*>(b + o_nt);
@@ -221,8 +222,6 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.wchunk_row0 = reinterpret_cast<int32_t*>(b + o_wr);
   c->pp.wchunk_rows = reinterpret_cast<int32_t*>(b + o_wn);
   c->pp.n_wchunks = reinterpret_cast<int32_t*>(b + o_nw);
-  c->pp.slot_to_prow = reinterpret_cast<int32_t*>(b + o_s2p);
-  c->pp.prow_to_slot = reinterpret_cast<int32_t*>(b + o_p2s);
   c->pp.blk_prefix = reinterpret_cast<int32_t*>(b + o_bp);
   c->pp.ticket = reinterpret_cast<unsigned int*>(b + o_tk);
   c->pp.tile_counter = c->pp.ticket + 4;   // same 256-byte slot
@@ -254,10 +253,15 @@ int grouter_plan(grouter_ctx* ctx, const void* idx, const int32_t* fold_map, int
     return GROUTER_ERR_MISALIGNED;
   if (!fold_map && ctx->dims.E_src != ctx->dims.E_tgt) return GROUTER_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  for (int phase = 0; phase < 2; ++phase) {
-    Timed tm(ctx, phase, st);
+  static const int slot_of_phase[PLAN_PHASES] = {0, 13, 1};
+  for (int phase = 0; phase < PLAN_PHASES; ++phase) {
+    Timed tm(ctx, slot_of_phase[phase], st);
     if (launch_plan(ctx, phase, idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
+  // fwd and bwd read the permutation from the caller's arrays
+  ctx->pp.offsets = offsets;
+  ctx->pp.row_to_slot = row_to_slot;
+  ctx->pp.slot_to_row = slot_to_row;
   ctx->planned = true;
   ctx->forwarded = false;
   return GROUTER_OK;

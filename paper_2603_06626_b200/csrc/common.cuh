@@ -24,32 +24,48 @@ constexpr int GEMM_CYCLE_COUNTERS = 5;   // issuer cycles, cycles waiting for op
 constexpr int WCHUNK_SPLIT = 1 << 30; // flag in PaddedPlan::wchunk_expert: the expert has several chunks
 constexpr int PLAN_THREADS = 256;    // 8 warps per plan block
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
-constexpr int PLAN_MIN_CHUNK = 2048; // slots per plan block (lower bound)
-constexpr int PLAN_MAX_BLOCKS = 1184;// 148 SMs x 8 resident blocks
+// Two forms of the plan kernels.  The counted form (E_tgt <= 256 and a fold table that fits shared memory) gives every
+// thread a run of `ipt` consecutive slots and a private counter per expert; the ballot form serves everything else.
+constexpr int PLAN_COUNTED_MAX_E = 256;
+constexpr int PLAN_COUNTED_MAX_ESRC = 4096;
+constexpr int PLAN_MIN_CHUNK = 2048; // ballot form: slots per plan block (lower bound)
+constexpr int PLAN_MAX_BLOCKS = 1184;// ballot form: 148 SMs x 8 resident blocks
 
 struct PlanGeom {
   int chunk;    // slots per block, multiple of 256
   int nblk;     // blocks
+  int ipt;      // counted form: consecutive slots per thread (16, 32 or 64); 0 = ballot form
 };
 
-inline PlanGeom plan_geom(int64_t R) {
-  int64_t chunk = (R + PLAN_MAX_BLOCKS - 1) / PLAN_MAX_BLOCKS;
-  if (chunk < PLAN_MIN_CHUNK) chunk = PLAN_MIN_CHUNK;
-  chunk = (chunk + PLAN_THREADS - 1) / PLAN_THREADS * PLAN_THREADS;
+inline PlanGeom plan_geom(int64_t R, int E_src, int E_tgt) {
   PlanGeom g;
-  g.chunk = (int)chunk;
-  g.nblk = (int)((R + chunk - 1) / chunk);
+  if (E_tgt <= PLAN_COUNTED_MAX_E && E_src <= PLAN_COUNTED_MAX_ESRC) {
+    // short runs while the problem is small (more blocks in flight), long ones once every SM has several blocks anyway
+    // (the per-block scan of the counters costs the same whatever the run length)
+    g.ipt = R <= (1 << 20) ? 16 : R <= (1 << 22) ? 32 : 64;
+    g.chunk = g.ipt * PLAN_THREADS;
+  } else {
+    int64_t chunk = (R + PLAN_MAX_BLOCKS - 1) / PLAN_MAX_BLOCKS;
+    if (chunk < PLAN_MIN_CHUNK) chunk = PLAN_MIN_CHUNK;
+    chunk = (chunk + PLAN_THREADS - 1) / PLAN_THREADS * PLAN_THREADS;
+    g.ipt = 0;
+    g.chunk = (int)chunk;
+  }
+  g.nblk = (int)((R + g.chunk - 1) / g.chunk);
   if (g.nblk < 1) g.nblk = 1;
   return g;
 }
 
-// Device-side copy of the plan in the 128-row-padded layout the GEMMs use.
+// What the context keeps of the plan: the 128-row-padded layout the GEMMs use and their work lists.  The
+// permutation itself stays in the caller's arrays (row_to_slot, slot_to_row, offsets), which fwd and bwd read:
+// padded row = row + row_shift[expert of the row].
 struct PaddedPlan {
   int32_t* pad_offsets;   // [E_tgt+1] first padded row of each expert; [E_tgt] = rows in use
   int32_t* row_shift;     // [E_tgt]   pad_offsets[e] - offsets[e]
   int32_t* pad_begin;     // [E_tgt]   first pad row of expert e (pad_offsets[e] + counts[e])
   // Tile list of the row-parallel GEMMs.  A tile is 256 rows of one expert (two 128-row halves, one per CTA
   // of a pair); an expert with an odd number of 128-row blocks ends in a tile whose second half is unused.
+  int32_t* pair_prefix;   // [E_tgt+1] exclusive prefix of 256-row tiles per expert
   int32_t* pair_row0;     // [max_m_tiles] first padded row of each 256-row tile
   int32_t* pair_expert;   // [max_m_tiles] expert of the tile; bit 30 set when the second half holds rows of that expert
   int32_t* n_pair_tiles;  // [1]
@@ -59,13 +75,15 @@ struct PaddedPlan {
   int32_t* wchunk_row0;   // [max_wchunks] first padded row of the chunk
   int32_t* wchunk_rows;   // [max_wchunks] rows in the chunk (multiple of 64; 0 for an expert without slots)
   int32_t* n_wchunks;     // [1]
-  int32_t* slot_to_prow;  // [R]
-  int32_t* prow_to_slot;  // [R_pad_max], -1 on pad rows
   int32_t* blk_prefix;    // [E_tgt * nblk] per-block histogram, then exclusive prefix over blocks
   unsigned int* ticket;   // [1] last-block-done counter
   int wgrad_chunk_blocks;       // longest weight-gradient chunk, in row tiles
   unsigned int* tile_counter;   // [1] next tile of the running grouped GEMM; zero between launches
   int32_t* status;        // [1] sticky status bits
+  // the caller's plan arrays of the latest grouter_plan (device pointers; valid until the caller overwrites them)
+  const int32_t* offsets;      // [E_tgt+1]
+  const int32_t* row_to_slot;  // [R]
+  const int32_t* slot_to_row;  // [R]
 };
 
 }  // namespace grouter
@@ -115,12 +133,14 @@ struct Workspace {
 Workspace carve_workspace(const grouter_dims& dm, int64_t R_pad_max, void* base);
 
 // ---- launchers (each returns a cudaError_t from the launch) ----
+// phase 0: per-block histograms; 1: prefixes over blocks, offsets, padded layout, work lists; 2: stable permutation, tile list
+constexpr int PLAN_PHASES = 3;
 cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
                         int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st);
 
-// dst[prow,:] = src[slot/k,:] for every routed slot; pad rows zero-filled.
+// dst[prow,:] = src[slot/k,:] for every routed slot (prow = slot_to_row[slot] + row_shift[expert]); pad rows zero-filled.
 cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st);
-// out[t,:] = sum_j src[slot_to_prow[t*k+j],:] (fp32 sum in slot order); optionally
+// out[t,:] = sum_j src[prow(t*k+j),:] (fp32 sum in slot order); optionally
 // dgates[t,j] = sum_n dgate_part[n][prow].
 cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part,
                                int n_part, float* dgates, cudaStream_t st);

@@ -64,7 +64,9 @@ struct GemmParams {
   int32_t tiles_m, tiles_n;    // output tiles per problem (tiles_m unused by row-parallel modes)
   int64_t R_pad_max;
   // epilogue
-  const int32_t* prow_to_slot;
+  const int32_t* row_to_slot;  // the plan's inverse permutation (unpadded rows)
+  const int32_t* row_shift;    // [E] padded row - row, per expert
+  const int32_t* pad_begin;    // [E] first pad row of each expert's padded segment
   const void* gates;
   int32_t gate_is_f32;
   const __nv_bfloat16* in_G;   // DH
@@ -181,9 +183,10 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
   return ti;
 }
 
-__device__ __forceinline__ float gate_of_row(const GemmParams& p, int prow) {
-  const int slot = __ldg(p.prow_to_slot + prow);
-  if (slot < 0) return 0.f;
+// Gate of padded row `prow` of expert e (0 on a pad row): the slot is row_to_slot[prow - row_shift[e]].
+__device__ __forceinline__ float gate_of_row(const GemmParams& p, int e, int prow) {
+  if (prow >= __ldg(p.pad_begin + e)) return 0.f;
+  const int slot = __ldg(p.row_to_slot + (prow - __ldg(p.row_shift + e)));
   if (p.gate_is_f32) return __ldg(reinterpret_cast<const float*>(p.gates) + slot);
   return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.gates)[slot]);
 }
@@ -529,7 +532,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (MODE == MODE_UP) {
         // accumulator columns 0..127 = gate, 128..255 = up, for F-columns col0..col0+127; this warp: 64 of them
         if (live && ti.n_valid - half * 64 > 0) {
-          const float g = gate_of_row(p, ti.row0 + r);
+          const float g = gate_of_row(p, ti.e, ti.row0 + r);
           const int x = ti.col0 + half * 64;
           uint32_t ph[32];                 // H' of the 64 columns, packed bf16 pairs
 #pragma unroll
@@ -585,7 +588,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       } else if (MODE == MODE_DH) {
-        const float g = live ? gate_of_row(p, ti.row0 + r) : 0.f;
+        const float g = live ? gate_of_row(p, ti.e, ti.row0 + r) : 0.f;
         float dgate = 0.f;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {                // four 32-column chunks; chunks 2c, 2c+1 fill one pair of blocks
@@ -785,7 +788,9 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.F = F;
   p.R_pad_max = ctx->R_pad_max;
   p.accumulate = (dm.flags & GROUTER_FLAG_ACCUMULATE_DW) ? 1 : 0;
-  p.prow_to_slot = ctx->pp.prow_to_slot;
+  p.row_to_slot = ctx->pp.row_to_slot;
+  p.row_shift = ctx->pp.row_shift;
+  p.pad_begin = ctx->pp.pad_begin;
   p.gates = gates;
   p.gate_is_f32 = dm.gate_dtype == GROUTER_GATE_F32;
   p.status = ctx->pp.status;

@@ -4,8 +4,10 @@
 // token row is read (scatter) or written (reduce) exactly once and every
 // routed row is touched exactly once: (T + R) * d * 2 bytes, the algorithmic
 // minimum.
-//   scatter_rows: dst[slot_to_prow[t*k+j], :] = src[t, :]      (gather of X / dY)
-//   reduce_rows : out[t, :] = sum_j src[slot_to_prow[t*k+j], :]  (Eq. 1 combine; dX)
+//   scatter_rows: dst[prow(t*k+j), :] = src[t, :]      (gather of X / dY)
+//   reduce_rows : out[t, :] = sum_j src[prow(t*k+j), :]  (Eq. 1 combine; dX)
+// prow(s) = slot_to_row[s] + row_shift[e], e the expert whose segment holds the row (found by bisection of the
+// offsets, which every block keeps in shared memory): the plan stores the permutation once, unpadded.
 // The gate weights are already folded into the rows by the GEMM epilogues, so
 // the combine is an unweighted fp32 sum in slot order (deterministic).
 #include "common.cuh"
@@ -26,18 +28,43 @@ __device__ __forceinline__ void st_v4(void* p, const uint4& v) {
   asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+constexpr int MAX_EXPERTS = 1024;
+
+// Offsets and row shifts into shared memory (E + 1 and E entries).
+__device__ __forceinline__ void load_layout(const int32_t* __restrict__ offsets, const int32_t* __restrict__ row_shift, int E,
+                                            int32_t* s_off, int32_t* s_shift) {
+  for (int e = threadIdx.x; e <= E; e += blockDim.x) {
+    s_off[e] = __ldg(offsets + e);
+    if (e < E) s_shift[e] = __ldg(row_shift + e);
+  }
+  __syncthreads();
+}
+// Padded row of routed row `row`: its expert is the last e with offsets[e] <= row (never an expert without rows).
+__device__ __forceinline__ int padded_row(int row, const int32_t* s_off, const int32_t* s_shift, int E) {
+  int lo = 0, hi = E;  // invariant: s_off[lo] <= row < s_off[hi]
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (s_off[mid] <= row) lo = mid; else hi = mid;
+  }
+  return row + s_shift[lo];
+}
+
 // SEG: 16-byte units each lane holds per pass; a warp moves SEG * 512 contiguous bytes of a row at a time.
 template <int SEG>
 __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
-                                                                    const int32_t* __restrict__ slot_to_prow,
+                                                                    const int32_t* __restrict__ slot_to_row,
+                                                                    const int32_t* __restrict__ offsets,
+                                                                    const int32_t* __restrict__ row_shift,
                                                                     const int32_t* __restrict__ pad_begin,
                                                                     const int32_t* __restrict__ pad_offsets, int T, int k, int d, int E) {
+  __shared__ int32_t s_off[MAX_EXPERTS + 1], s_shift[MAX_EXPERTS];
+  load_layout(offsets, row_shift, E, s_off, s_shift);
   const int lane = threadIdx.x & 31;
   const int gwarp = blockIdx.x * MOVE_WARPS + (threadIdx.x >> 5);
   const int nwarps = gridDim.x * MOVE_WARPS;
   const int units = d >> 3;  // 16-byte units per row
   for (int t = gwarp; t < T; t += nwarps) {
-    const int my_prow = lane < k ? __ldg(slot_to_prow + (size_t)t * k + lane) : 0;
+    const int my_prow = lane < k ? padded_row(__ldg(slot_to_row + (size_t)t * k + lane), s_off, s_shift, E) : 0;
     const char* s = reinterpret_cast<const char*>(src + (size_t)t * d);
     for (int u0 = 0; u0 < units; u0 += 32 * SEG) {
       uint4 v[SEG];
@@ -82,15 +109,19 @@ __device__ __forceinline__ void acc_bf16x8(float (&a)[8], const uint4& v) {
 // before it moves to the next row, so DRAM sees long sequential bursts instead of many interleaved short ones.
 template <int SEG>
 __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ out,
-                                                                   const int32_t* __restrict__ slot_to_prow, int T, int k, int d,
+                                                                   const int32_t* __restrict__ slot_to_row,
+                                                                   const int32_t* __restrict__ offsets,
+                                                                   const int32_t* __restrict__ row_shift, int T, int k, int d, int E,
                                                                    const float* __restrict__ dgate_part, int n_part, size_t part_stride,
                                                                    float* __restrict__ dgates) {
+  __shared__ int32_t s_off[MAX_EXPERTS + 1], s_shift[MAX_EXPERTS];
+  load_layout(offsets, row_shift, E, s_off, s_shift);
   const int lane = threadIdx.x & 31;
   const int gwarp = blockIdx.x * MOVE_WARPS + (threadIdx.x >> 5);
   const int nwarps = gridDim.x * MOVE_WARPS;
   const int units = d >> 3;
   for (int t = gwarp; t < T; t += nwarps) {
-    const int my_prow = lane < k ? __ldg(slot_to_prow + (size_t)t * k + lane) : 0;
+    const int my_prow = lane < k ? padded_row(__ldg(slot_to_row + (size_t)t * k + lane), s_off, s_shift, E) : 0;
     if (dgates != nullptr && lane < k) {
       float g = 0.f;
       for (int n = 0; n < n_part; ++n) g += dgate_part[(size_t)n * part_stride + my_prow];
@@ -156,16 +187,16 @@ static int mover_grid(const grouter_ctx* ctx, int T) {
 
 cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  scatter_rows_kernel<SCATTER_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_prow, ctx->pp.pad_begin,
-                                                                      ctx->pp.pad_offsets, dm.T, dm.k, dm.d, dm.E_tgt);
+  scatter_rows_kernel<SCATTER_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift,
+                                                                      ctx->pp.pad_begin, ctx->pp.pad_offsets, dm.T, dm.k, dm.d, dm.E_tgt);
   return cudaGetLastError();
 }
 
 cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part, int n_part,
                                float* dgates, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  reduce_rows_kernel<REDUCE_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_prow, dm.T, dm.k, dm.d, dgate_part, n_part,
-                                                                     (size_t)ctx->R_pad_max, dgates);
+  reduce_rows_kernel<REDUCE_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift, dm.T, dm.k, dm.d,
+                                                                     dm.E_tgt, dgate_part, n_part, (size_t)ctx->R_pad_max, dgates);
   return cudaGetLastError();
 }
 

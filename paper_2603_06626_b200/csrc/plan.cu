@@ -1,23 +1,436 @@
 // Routing-plan build: a stable counting sort of the R = T*k slots by target
-// expert, in two launches.
+// expert, in three launches.
 //
-//   plan_hist_kernel    every block histograms a contiguous chunk of slots
-//                       (one private histogram per warp, built from warp
-//                       ballots so no atomics are needed); the last
-//                       block to finish turns the per-block histograms into
-//                       exclusive prefixes over blocks, scans the expert
-//                       counts into offsets, and lays out the 128-row-padded
-//                       segments and the tile list the grouped GEMMs walk.
-//   plan_permute_kernel every warp walks its sub-chunk in slot order; the rank
-//                       of a slot among equal experts is (block prefix) +
-//                       (earlier warps of the block) + (earlier lanes), which
-//                       makes the permutation stable and bit-reproducible.
+//   phase 0  per-block histograms       every block counts the experts of a contiguous chunk of slots
+//   phase 1  scans and layout           one block per expert turns its row of per-block counts into exclusive
+//                                       prefixes over blocks; the last block to finish scans the expert totals into
+//                                       offsets, lays out the 128-row-padded segments and orders the work list of
+//                                       the weight-gradient GEMMs
+//   phase 2  stable permutation         rank of a slot among equal experts = (earlier blocks) + (earlier slots of
+//                                       this block); also writes the tile list of the row-parallel GEMMs
+//
+// Phases 0 and 2 come in two forms.
+//   counted (E_tgt <= 256, fold table in shared memory): a thread owns a run of 16-64 consecutive slots, fetched with
+//     16-byte loads, and a private 16-bit counter per expert in shared memory (no atomics, no warp votes).  A scan over
+//     the threads' counters gives every thread its first rank per expert; the thread then walks its run once more,
+//     handing out ranks in slot order.  The rows go to slot_to_row directly (a thread's run is contiguous there);
+//     the inverse goes through a shared-memory staging array ordered by (expert, rank), so row_to_slot is written in
+//     contiguous runs, one per expert and block.
+//   ballot (any E_tgt up to 1024, any E_src): a warp walks its sub-chunk 32 slots at a time; lanes with equal keys are
+//     found with one vote per key bit.
+// Both are bit-reproducible: no result depends on the order in which threads or blocks run.
 //
 // The fold map is the compact form of the paper's binary folding matrix M
 // (section "Expert Folding"): e_s = fold_map[idx_s].
 #include "common.cuh"
 
 namespace grouter {
+
+__device__ __forceinline__ int bits_for(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
+
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Counted form
+// ------------------------------------------------------------------------------------------------------------------
+
+// How raw ids become target experts.  `table` (shared memory, one 16-bit entry per source id) holds the fold target, or
+// 0x8000 for a target outside [0, E_tgt); without a fold map the id is the target.
+struct FoldView {
+  const uint16_t* table;   // null: identity
+  int E_src;
+  bool plain;              // 8-bit ids, no fold map, E_src == 256: every byte is a valid target as it stands
+};
+
+__device__ __forceinline__ uint32_t fold_one(uint32_t raw, const FoldView& f, int& bad) {
+  if (raw >= (uint32_t)f.E_src) {
+    bad = 1;
+    raw = 0;
+  }
+  if (f.table == nullptr) return raw;
+  const uint32_t t = f.table[raw];
+  if (t & 0x8000u) bad = 1;
+  return t & 0xffu;
+}
+
+// Target experts of the 16 slots s .. s+15 as 16 bytes (slot s+i in byte i); slots at or beyond R read as 0 and are
+// not checked.  s is a multiple of 16 and idx is 16-byte aligned, so every 16-byte load is aligned and holds at least
+// one valid id: it cannot leave the page the ids end in.
+template <typename IdxT>
+__device__ __forceinline__ uint4 load_targets16(const IdxT* __restrict__ idx, int s, int R, const FoldView& f, int& bad) {
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  if (sizeof(IdxT) == 1) {
+    if (s < R) {
+      const uint4 v = ld_nc_v4(reinterpret_cast<const uint8_t*>(idx) + s);
+      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    }
+    if (!f.plain) {
+      const int n = min(16, max(0, R - s));
+      // without a fold map a valid id is its own target: test four bytes at once for id >= E_src (bit 7 of a byte of
+      // `over`), and take the byte-by-byte path only for a word that holds a bad id, a fold table, or the ragged end
+      const uint32_t add = (uint32_t)((f.E_src <= 128 ? 128 - f.E_src : 256 - f.E_src) * 0x01010101);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (f.table == nullptr && q * 4 + 4 <= n) {
+          const uint32_t t = ((w[q] & 0x7f7f7f7fu) + add) & 0x80808080u;     // low seven bits reach the bound
+          const uint32_t over = f.E_src <= 128 ? (t | (w[q] & 0x80808080u)) : (t & w[q]);
+          if (over == 0u) continue;
+        }
+        uint32_t o = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+          if (q * 4 + b < n) o |= fold_one((w[q] >> (8 * b)) & 0xffu, f, bad) << (8 * b);
+        w[q] = o;
+      }
+    }
+  } else {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (s + 4 * q < R) {
+        const uint4 v = ld_nc_v4(reinterpret_cast<const int32_t*>(idx) + s + 4 * q);
+        const uint32_t r[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+          if (s + 4 * q + b < R) o |= fold_one(r[b], f, bad) << (8 * b);
+        w[q] = o;
+      }
+    }
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Fold table into shared memory (one thread per entry, strided); returns the view the item loops use.
+template <typename IdxT>
+__device__ __forceinline__ FoldView make_fold_view(const int32_t* __restrict__ fold_map, int E_src, int E_tgt, uint16_t* s_fold) {
+  FoldView f;
+  f.E_src = E_src;
+  f.table = fold_map ? s_fold : nullptr;
+  f.plain = sizeof(IdxT) == 1 && fold_map == nullptr && E_src == 256;
+  if (fold_map)
+    for (int i = threadIdx.x; i < E_src; i += PLAN_THREADS) {
+      const int t = __ldg(fold_map + i);
+      s_fold[i] = (unsigned)t < (unsigned)E_tgt ? (uint16_t)t : (uint16_t)0x8000u;
+    }
+  return f;
+}
+
+// Private counters of the counted form.  Every thread keeps one 16-bit counter per expert in shared memory; threads t
+// and t + 128 share the 32-bit word [e][t & 127] (low and high half), so the 32 lanes of a warp always touch 32
+// different banks whatever their experts are, and a counter's address is e * 512 + a per-thread constant.  A thread
+// reads and writes only its own halves (16-bit accesses), so nothing needs an atomic: shared-memory atomics cost about
+// ten cycles per warp instruction here, conflict-free or not, which made both walks slower than plain loads and stores.
+// To keep several loads in flight the walks take four slots at a time: four loads, then the ranks are corrected in
+// registers for equal experts among the four, then four stores in slot order (a later store of the same counter holds
+// the larger value).  No half can overflow: every value stays at or below the block's slot count (at most 16384).
+constexpr int CNT_ROW_WORDS = PLAN_THREADS / 2;     // words per expert row
+
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+}
+// Shared-memory address of this thread's counter of expert 0; the one of expert e lies e * 512 bytes further.
+__device__ __forceinline__ uint32_t my_counters(const uint32_t* s_cnt) {
+  return (uint32_t)__cvta_generic_to_shared(s_cnt) + 4u * (threadIdx.x & (CNT_ROW_WORDS - 1)) + (threadIdx.x >= CNT_ROW_WORDS ? 2u : 0u);
+}
+// Four slots (experts in the bytes of w, slot order = byte order; only the first n are real): bumps their counters and
+// returns the values the counters held before each slot's own bump.
+__device__ __forceinline__ void bump4(uint32_t mine, uint32_t w, int n, uint32_t (&before)[4]) {
+  const uint32_t a0 = mine + ((w & 0xffu) << 9), a1 = mine + ((w & 0xff00u) << 1), a2 = mine + ((w & 0xff0000u) >> 7),
+                 a3 = mine + ((w >> 24) << 9);
+  uint32_t c0 = lds_u16(a0), c1 = lds_u16(a1), c2 = lds_u16(a2), c3 = lds_u16(a3);
+  c1 += (a1 == a0);
+  c2 += (a2 == a0) + (a2 == a1);
+  c3 += (a3 == a0) + (a3 == a1) + (a3 == a2);
+  before[0] = c0; before[1] = c1; before[2] = c2; before[3] = c3;
+  if (n >= 4) {
+    sts_u16(a0, c0 + 1u);
+    sts_u16(a1, c1 + 1u);
+    sts_u16(a2, c2 + 1u);
+    sts_u16(a3, c3 + 1u);
+  } else {
+    if (n > 0) sts_u16(a0, c0 + 1u);
+    if (n > 1) sts_u16(a1, c1 + 1u);
+    if (n > 2) sts_u16(a2, c2 + 1u);
+  }
+}
+
+// Tile list of the row-parallel GEMMs, written by the threads of phase 2 before they start on the permutation:
+// expert and first padded row of every 256-row tile.  The last e with pair_prefix[e] <= t owns tile t.
+// s_pp / s_po: shared-memory copies of pair_prefix and pad_offsets, E_tgt + 1 entries each.
+__device__ __forceinline__ void write_tile_list(const PaddedPlan& pp, int E_tgt, int32_t* s_pp, int32_t* s_po) {
+  for (int e = threadIdx.x; e <= E_tgt; e += PLAN_THREADS) {
+    s_pp[e] = pp.pair_prefix[e];
+    s_po[e] = pp.pad_offsets[e];
+  }
+  __syncthreads();
+  const int n_tiles = s_pp[E_tgt];
+  for (int t = blockIdx.x * PLAN_THREADS + threadIdx.x; t < n_tiles; t += gridDim.x * PLAN_THREADS) {
+    int lo = 0, hi = E_tgt;  // invariant: s_pp[lo] <= t < s_pp[hi]
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_pp[mid] <= t) lo = mid; else hi = mid;
+    }
+    const int row0 = s_po[lo] + (t - s_pp[lo]) * 2 * ROW_TILE;
+    pp.pair_row0[t] = row0;
+    pp.pair_expert[t] = lo | (row0 + ROW_TILE < s_po[lo + 1] ? PAIR_VALID2 : 0);
+  }
+}
+
+// Phase 0, counted form: per-warp histograms with shared-memory adds (a word of four equal ids is one add of 4).
+// Shared-memory atomics cost about ten cycles per warp instruction here, with or without conflicts; private counters
+// as in phase 2 (no atomics, but 512 bytes of counters per expert to clear and to sum per block) were measured slower
+// for this kernel, which needs nothing but the block's totals.
+template <typename IdxT, int V>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_count_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                  int R, int E_src, int E_tgt, int nblk,
+                                                                  int32_t* __restrict__ blk_hist, int32_t* __restrict__ status) {
+  constexpr int IPT = 16 * V;
+  constexpr int CHUNK = IPT * PLAN_THREADS;
+  extern __shared__ __align__(16) uint32_t sm_u32[];
+  uint32_t* s_hist = sm_u32;                                                       // [PLAN_WARPS][E_tgt]
+  uint16_t* s_fold = reinterpret_cast<uint16_t*>(sm_u32 + PLAN_WARPS * E_tgt);     // [E_src]
+  const int tid = threadIdx.x, warp = tid >> 5;
+  for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) s_hist[i] = 0u;
+  const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
+  __syncthreads();
+  uint32_t* h = s_hist + warp * E_tgt;
+  const int s0 = blockIdx.x * CHUNK + tid * IPT;
+  const int n_mine = min(IPT, max(0, R - s0));
+  int bad = 0;
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    const uint4 ev = load_targets16<IdxT>(idx, s0 + 16 * v, R, f, bad);
+    const uint32_t w[4] = {ev.x, ev.y, ev.z, ev.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int nq = n_mine - (16 * v + 4 * q);
+      if (nq >= 4 && w[q] == __byte_perm(w[q], 0u, 0x0321)) {
+        atomicAdd(h + (w[q] & 0xffu), 4u);
+      } else {
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+          if (b < nq) atomicAdd(h + ((w[q] >> (8 * b)) & 0xffu), 1u);
+      }
+    }
+  }
+  if (bad) atomicOr(status, STATUS_BAD_INDEX);
+  __syncthreads();
+  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+    uint32_t tot = 0u;
+#pragma unroll
+    for (int w = 0; w < PLAN_WARPS; ++w) tot += s_hist[w * E_tgt + e];
+    blk_hist[(size_t)e * nblk + blockIdx.x] = (int32_t)tot;
+  }
+}
+
+constexpr int PLACE_BIG_RUN = 1024;   // an expert with more slots than this in one block is copied out by the whole block
+
+// Shared-memory layout of plan_place_kernel, in bytes from the start of the dynamic block.
+struct PlaceSmem {
+  int cnt, stage, first, tot, big, fold, pp, po, bytes;
+};
+__host__ __device__ inline PlaceSmem place_smem(int E_src, int E_tgt, int ipt, bool with_fold) {
+  PlaceSmem m;
+  int off = 0;
+  auto take = [&](int n) { const int o = off; off += (n + 15) / 16 * 16; return o; };
+  const int cnt_bytes = E_tgt * CNT_ROW_WORDS * 4, row_bytes = ipt * PLAN_THREADS * 4;
+  m.cnt = take(cnt_bytes > row_bytes ? cnt_bytes : row_bytes);   // private counters; afterwards the row of every slot of the chunk
+  m.stage = take(ipt * PLAN_THREADS * 2);       // slot (as its index within the chunk) at every (expert, rank) position
+  m.first = take(E_tgt * 8);                    // per expert {first staging position, first global row of this block}
+  m.tot = take(E_tgt * 4);                      // per expert: slots in this block
+  m.big = take((E_tgt + 1) * 4);                // [0] = how many, then the experts with more than PLACE_BIG_RUN slots here
+  m.fold = take(with_fold ? E_src * 2 : 0);
+  m.pp = take((E_tgt + 1) * 4);
+  m.po = take((E_tgt + 1) * 4);
+  m.bytes = off;
+  return m;
+}
+
+// Phase 2, counted form.
+template <typename IdxT, int V>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_place_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                  int R, int E_src, int E_tgt, int nblk, PaddedPlan pp,
+                                                                  const int32_t* __restrict__ offsets, int32_t* __restrict__ row_to_slot,
+                                                                  int32_t* __restrict__ slot_to_row) {
+  constexpr int IPT = 16 * V;
+  constexpr int CHUNK = IPT * PLAN_THREADS;
+  static_assert(CHUNK <= 32768, "ranks within a block are kept in 16 bits, two to a word");
+  extern __shared__ __align__(16) uint8_t sm_raw[];
+  const PlaceSmem L = place_smem(E_src, E_tgt, IPT, fold_map != nullptr);
+  uint32_t* s_cnt = reinterpret_cast<uint32_t*>(sm_raw + L.cnt);
+  uint16_t* s_stage = reinterpret_cast<uint16_t*>(sm_raw + L.stage);
+  int32_t* s_rows = reinterpret_cast<int32_t*>(sm_raw + L.cnt);     // the counters' space, once they are no longer needed
+  int2* s_first = reinterpret_cast<int2*>(sm_raw + L.first);
+  int32_t* s_tot = reinterpret_cast<int32_t*>(sm_raw + L.tot);
+  int32_t* s_big = reinterpret_cast<int32_t*>(sm_raw + L.big);
+  uint16_t* s_fold = reinterpret_cast<uint16_t*>(sm_raw + L.fold);
+  __shared__ int s_warp_sum[PLAN_WARPS];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  write_tile_list(pp, E_tgt, reinterpret_cast<int32_t*>(sm_raw + L.pp), reinterpret_cast<int32_t*>(sm_raw + L.po));
+
+  {
+    uint4* z = reinterpret_cast<uint4*>(s_cnt);
+    for (int i = tid; i < E_tgt * CNT_ROW_WORDS / 4; i += PLAN_THREADS) z[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
+  // Per expert (E_tgt <= 256 = one per thread): this block's slot count, from the prefixes over blocks that phase 1
+  // left; its exclusive scan over experts = the expert's first position in the staging array; the first global row.
+  {
+    const int e = tid;
+    int cnt = 0, before = 0;
+    if (e < E_tgt) {
+      const int32_t* rowp = pp.blk_prefix + (size_t)e * nblk + blockIdx.x;
+      before = __ldcg(rowp);
+      const int next = blockIdx.x + 1 < nblk ? __ldcg(rowp + 1) : __ldg(offsets + e + 1) - __ldg(offsets + e);
+      cnt = next - before;
+    }
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    if (lane == 31) s_warp_sum[warp] = incl;
+    if (tid == 0) s_big[0] = 0;
+    __syncthreads();
+    int start = incl - cnt;
+#pragma unroll
+    for (int w = 0; w < PLAN_WARPS; ++w)
+      if (w < warp) start += s_warp_sum[w];
+    if (e < E_tgt) {
+      const int first_row = __ldg(offsets + e) + before;
+      s_first[e] = make_int2(start, first_row);
+      s_tot[e] = cnt;
+      if (cnt > PLACE_BIG_RUN) s_big[1 + atomicAdd(&s_big[0], 1)] = e;
+    }
+  }
+
+  // ---- first walk: count this thread's slots per expert ----
+  const int chunk0 = blockIdx.x * CHUNK;
+  const int s0 = chunk0 + tid * IPT;
+  const int n_mine = min(IPT, max(0, R - s0));
+  const uint32_t mine = my_counters(s_cnt);
+  uint4 ev[V];
+  int bad = 0;
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    ev[v] = load_targets16<IdxT>(idx, s0 + 16 * v, R, f, bad);
+    const uint32_t w[4] = {ev[v].x, ev[v].y, ev[v].z, ev[v].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t before[4];
+      const int n = n_mine - (16 * v + 4 * q);
+      if (n > 0) bump4(mine, w[q], n, before);
+    }
+  }
+  if (bad) atomicOr(pp.status, STATUS_BAD_INDEX);
+  __syncthreads();
+
+  // ---- exclusive scan over the threads, one expert row per warp at a time; the result starts at the expert's first
+  // staging position, so a counter then holds the staging position of its thread's next slot of that expert ----
+  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
+    uint4* rowp = reinterpret_cast<uint4*>(s_cnt + e * CNT_ROW_WORDS) + lane;    // threads 4*lane .. +3 (low) and 128 + 4*lane .. (high)
+    const uint4 a = *rowp;
+    const uint32_t sum = a.x + a.y + a.z + a.w;
+    uint32_t incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += n;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    const uint32_t start = (uint32_t)s_first[e].x;
+    // low halves count from `start`, high halves (threads 128..255) from start + (slots of threads 0..127)
+    const uint32_t x0 = incl - sum + (start | ((start + (total & 0xffffu)) << 16));
+    const uint32_t x1 = x0 + a.x, x2 = x1 + a.y, x3 = x2 + a.z;
+    *rowp = make_uint4(x0, x1, x2, x3);
+  }
+  __syncthreads();
+
+  // ---- second walk: hand out the positions in slot order ----
+  const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(s_stage);
+#pragma unroll
+  for (int v = 0; v < V; ++v) {
+    const uint32_t w[4] = {ev[v].x, ev[v].y, ev[v].z, ev[v].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i0 = 16 * v + 4 * q;
+      const int n = n_mine - i0;
+      if (n <= 0) continue;
+      uint32_t pos[4];
+      bump4(mine, w[q], n, pos);
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        if (b < n) sts_u16(stage_addr + 2u * pos[b], (uint32_t)(tid * IPT + i0 + b));
+    }
+  }
+  __syncthreads();
+
+  // ---- every expert's run of this block is contiguous in the staging array and in row_to_slot: the inverse permutation
+  // goes out in runs; the row of every slot is parked in shared memory (the counters are done with) ----
+  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
+    const int n = s_tot[e];
+    if (n > PLACE_BIG_RUN) continue;
+    const int2 t = s_first[e];
+    const uint16_t* src = s_stage + t.x;
+    int32_t* dst = row_to_slot + t.y;
+    int i = lane;
+    for (; i + 96 < n; i += 128) {
+      const int a = src[i], b = src[i + 32], c = src[i + 64], d = src[i + 96];
+      dst[i] = chunk0 + a;
+      dst[i + 32] = chunk0 + b;
+      dst[i + 64] = chunk0 + c;
+      dst[i + 96] = chunk0 + d;
+      s_rows[a] = t.y + i;
+      s_rows[b] = t.y + i + 32;
+      s_rows[c] = t.y + i + 64;
+      s_rows[d] = t.y + i + 96;
+    }
+    for (; i < n; i += 32) {
+      const int a = src[i];
+      dst[i] = chunk0 + a;
+      s_rows[a] = t.y + i;
+    }
+  }
+  const int n_big = s_big[0];
+  for (int j = 0; j < n_big; ++j) {
+    const int e = s_big[1 + j];
+    const int n = s_tot[e];
+    const int2 t = s_first[e];
+    for (int i = tid; i < n; i += PLAN_THREADS) {
+      const int a = s_stage[t.x + i];
+      row_to_slot[t.y + i] = chunk0 + a;
+      s_rows[a] = t.y + i;
+    }
+  }
+  __syncthreads();
+  // ---- slot_to_row: the chunk's rows, in slot order, as one contiguous copy ----
+  {
+    const int n_here = min(CHUNK, R - chunk0);
+    int32_t* dst = slot_to_row + chunk0;     // chunk0 is a multiple of 4096: 16-byte aligned
+    for (int i = 4 * tid; i < n_here; i += 4 * PLAN_THREADS) {
+      if (i + 4 <= n_here) {
+        *reinterpret_cast<int4*>(dst + i) = *reinterpret_cast<const int4*>(s_rows + i);
+      } else {
+        for (int j = i; j < n_here; ++j) dst[j] = s_rows[j];
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Ballot form
+// ------------------------------------------------------------------------------------------------------------------
 
 // Target expert of a raw id: range check, fold map, range check; a bad id or fold target counts as expert 0.
 __device__ __forceinline__ int fold_expert(int raw, const int32_t* __restrict__ fold_map, int E_src, int E_tgt, int32_t* status) {
@@ -46,7 +459,6 @@ __device__ __forceinline__ unsigned same_key_lanes(int key, int key_bits) {
   }
   return peers;
 }
-__device__ __forceinline__ int bits_for(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
 
 // Per-warp histograms of this block's chunk into hist[w*E + e] (smem, pre-zeroed).
 template <typename IdxT>
@@ -72,80 +484,88 @@ __device__ __forceinline__ void warp_histogram(const IdxT* __restrict__ idx, con
 }
 
 template <typename IdxT>
-__global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
-                                                                 int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
-                                                                 int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
-  extern __shared__ int32_t sm[];  // plan_hist_smem_ints(E) ints
-  __shared__ int s_last;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+__global__ void __launch_bounds__(PLAN_THREADS) plan_hist_ballot_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                        int R, int E_src, int E_tgt, int chunk, int nblk,
+                                                                        int32_t* __restrict__ blk_hist, int32_t* __restrict__ status) {
+  extern __shared__ int32_t sm[];  // PLAN_WARPS * E_tgt ints
+  const int tid = threadIdx.x;
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
   __syncthreads();
-  warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, pp.status);
+  warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, status);
   __syncthreads();
   for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
     int tot = 0;
 #pragma unroll
     for (int w = 0; w < PLAN_WARPS; ++w) tot += sm[w * E_tgt + e];
-    pp.blk_prefix[e * nblk + blockIdx.x] = tot;
+    blk_hist[(size_t)e * nblk + blockIdx.x] = tot;
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned t = atomicAdd(pp.ticket, 1u);
-    s_last = (t == (unsigned)(nblk - 1));
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+}
 
-  // ---- last block: prefixes over blocks, offsets, padded layout, tile list ----
+template <typename IdxT>
+__global__ void __launch_bounds__(PLAN_THREADS) plan_permute_ballot_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                           int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
+                                                                           const int32_t* __restrict__ offsets, int32_t* __restrict__ row_to_slot,
+                                                                           int32_t* __restrict__ slot_to_row) {
+  extern __shared__ int32_t sm[];  // PLAN_WARPS * E_tgt ints, then 2 * (E_tgt + 1) for the tile list
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  write_tile_list(pp, E_tgt, sm + PLAN_WARPS * E_tgt, sm + PLAN_WARPS * E_tgt + E_tgt + 1);
+  for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
+  __syncthreads();
+  warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, pp.status);
+  __syncthreads();
+  // per-warp histogram -> first row of (block, warp, expert)
+  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+    int base = offsets[e] + pp.blk_prefix[(size_t)e * nblk + blockIdx.x];
+#pragma unroll
+    for (int w = 0; w < PLAN_WARPS; ++w) {
+      const int t = sm[w * E_tgt + e];
+      sm[w * E_tgt + e] = base;
+      base += t;
+    }
+  }
+  __syncthreads();
+  const int wlen = chunk / PLAN_WARPS;
+  const int base = blockIdx.x * chunk + warp * wlen;
+  int32_t* cur = sm + warp * E_tgt;
+  const unsigned lt = (1u << lane) - 1u;
+  const int key_bits = bits_for(E_tgt);
+  int raw_next = (base + lane < R) ? (int)idx[base + lane] : 0;   // ids are fetched one iteration ahead
+  for (int i = 0; i < wlen; i += 32) {
+    const int s = base + i + lane;
+    const bool valid = s < R;
+    const int raw = raw_next;
+    if (i + 32 < wlen && s + 32 < R) raw_next = (int)idx[s + 32];
+    const int e = valid ? fold_expert(raw, fold_map, E_src, E_tgt, pp.status) : -1;
+    const unsigned mask = same_key_lanes(e, key_bits);
+    const int row = valid ? cur[e] + __popc(mask & lt) : 0;
+    __syncwarp();
+    if (valid && lane == 31 - __clz(mask)) cur[e] = row + 1;
+    __syncwarp();
+    if (valid) {
+      slot_to_row[s] = row;
+      row_to_slot[row] = s;
+    }
+    if (base + i + 32 >= R) break;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------------------------
+// Phase 1: prefixes over blocks, expert offsets, padded layout, work list of the weight gradients
+// ------------------------------------------------------------------------------------------------------------------
+static int plan_scan_smem_ints(int E) { return 11 * E + 4 + 2 * (WGRAD_LEN_BUCKETS + 1); }
+
+// Offsets, padded layout, tile prefix and the weight gradients' chunk list from the expert counts in s_cnt (= sm[0..E)).
+// Runs in one block of any size (a multiple of 32 threads); sm holds plan_scan_smem_ints(E_tgt) ints.
+__device__ __forceinline__ void plan_layout(int32_t* sm, int E_tgt, const PaddedPlan& pp, int32_t* __restrict__ counts,
+                                            int32_t* __restrict__ offsets) {
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nthr = blockDim.x, nwarps = blockDim.x >> 5;
   int32_t* s_cnt = sm;                    // [E]
   int32_t* s_off = sm + E_tgt;            // [E+1]
   int32_t* s_pad = sm + 2 * E_tgt + 1;    // [E+1]
   int32_t* s_pair = sm + 3 * E_tgt + 2;   // [E+1] exclusive prefix of 256-row tiles per expert
   int32_t* s_wch = sm + 4 * E_tgt + 3;    // [E+1] exclusive prefix of weight-gradient row chunks per expert
-  int32_t* s_wpos = sm + 5 * E_tgt + 4;   // [2E] list position of each expert's longer / shorter chunks, then [chunk lengths + 1]
-  __syncthreads();
-  // Exclusive prefix over blocks of every expert's per-block counts (row e of blk_prefix), and the expert totals.
-  // Eight lanes share one expert: each sums a contiguous segment of the row with its loads batched eight deep, the
-  // eight segment sums are scanned with shuffles, and a second sweep writes the running prefixes back.
-  {
-    const int grp = lane >> 3, gl = lane & 7;
-    const int seg = (nblk + 7) >> 3;
-    for (int e0 = warp * 4; e0 < E_tgt; e0 += PLAN_WARPS * 4) {
-      const int e = e0 + grp;
-      const bool have = e < E_tgt;
-      int32_t* rowp = pp.blk_prefix + (size_t)(have ? e : 0) * nblk;
-      const int b_lo = min(gl * seg, nblk), b_hi = have ? min(b_lo + seg, nblk) : b_lo;
-      int sum = 0;
-      for (int b = b_lo; b < b_hi; b += 8) {
-        int v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (b + j < b_hi) ? __ldcg(rowp + b + j) : 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) sum += v[j];
-      }
-      int incl = sum;
-#pragma unroll
-      for (int o = 1; o < 8; o <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, incl, o, 8);
-        if (gl >= o) incl += n;
-      }
-      int run = incl - sum;
-      for (int b = b_lo; b < b_hi; b += 8) {
-        int v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (b + j < b_hi) ? __ldcg(rowp + b + j) : 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (b + j < b_hi) rowp[b + j] = run;
-          run += v[j];
-        }
-      }
-      if (have && gl == 7) s_cnt[e] = incl;
-    }
-  }
-  __syncthreads();
+  int32_t* s_wpos = sm + 5 * E_tgt + 4;   // [2E] list position of each expert's longer / shorter chunks; the chunk-list arrays follow
+  __syncthreads();     // s_cnt is complete
   if (warp == 0) {
     const int per = (E_tgt + 31) / 32;
     const int e0 = min(lane * per, E_tgt), e1 = min(e0 + per, E_tgt);
@@ -193,74 +613,72 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
     }
   }
   __syncthreads();
-  for (int e = tid; e <= E_tgt; e += PLAN_THREADS) {
+  for (int e = tid; e <= E_tgt; e += nthr) {
     offsets[e] = s_off[e];
     pp.pad_offsets[e] = s_pad[e];
+    pp.pair_prefix[e] = s_pair[e];
     if (e < E_tgt) {
       counts[e] = s_cnt[e];
       pp.row_shift[e] = s_pad[e] - s_off[e];
       pp.pad_begin[e] = s_pad[e] + s_cnt[e];
     }
   }
-  const int n_tiles = s_pair[E_tgt];
   if (tid == 0) {
-    *pp.n_pair_tiles = n_tiles;
+    *pp.n_pair_tiles = s_pair[E_tgt];
     *pp.ticket = 0u;  // ready for the next plan
     *pp.tile_counter = 0u;  // a grouped GEMM that gave up on a timeout may have left it mid-count
-  }
-  // expert and first row of every 256-row tile: the last e with s_pair[e] <= t owns tile t
-  for (int t = tid; t < n_tiles; t += PLAN_THREADS) {
-    int lo = 0, hi = E_tgt;  // invariant: s_pair[lo] <= t < s_pair[hi]
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (s_pair[mid] <= t) lo = mid; else hi = mid;
-    }
-    const int row0 = s_pad[lo] + (t - s_pair[lo]) * 2 * ROW_TILE;
-    pp.pair_row0[t] = row0;
-    pp.pair_expert[t] = lo | (row0 + ROW_TILE < s_pad[lo + 1] ? PAIR_VALID2 : 0);
+    *pp.n_wchunks = s_wch[E_tgt];
   }
   // Row chunks of the weight-gradient GEMMs: an expert without slots keeps one empty chunk (its gradient is zero-filled).
   // An expert's blocks are cut into n chunks of near-equal size: `rem` chunks of base + 1 blocks, then n - rem of base.
   // The list is ordered by chunk length, longest first, in WGRAD_LEN_BUCKETS classes of length (within a class by
   // expert, then by position): tiles of similar cost are neighbours, and the shortest tiles at the end even out the tail.
-  if (tid == 0) *pp.n_wchunks = s_wch[E_tgt];
   {
     const int chunk_blocks = pp.wgrad_chunk_blocks;
     auto len_class = [chunk_blocks](int blocks) { return (blocks * WGRAD_LEN_BUCKETS + chunk_blocks - 1) / chunk_blocks; };   // 0 .. BUCKETS
-    // chunks of every class, then the first list position of every class (descending)
-    int32_t* s_len = s_wpos + 2 * E_tgt;   // [WGRAD_LEN_BUCKETS + 1]
-    for (int i = tid; i <= WGRAD_LEN_BUCKETS; i += PLAN_THREADS) s_len[i] = 0;
+    int32_t* s_c = s_wpos + 2 * E_tgt;                   // [2E] chunks of the expert's longer / shorter length
+    int32_t* s_cl = s_c + 2 * E_tgt;                     // [2E] their length classes
+    int32_t* s_len = s_cl + 2 * E_tgt;                   // [BUCKETS + 1] chunks per class
+    int32_t* s_start = s_len + WGRAD_LEN_BUCKETS + 1;    // [BUCKETS + 1] first list position of each class
+    for (int i = tid; i <= WGRAD_LEN_BUCKETS; i += nthr) s_len[i] = 0;
     __syncthreads();
-    for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+    for (int e = tid; e < E_tgt; e += nthr) {
       const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
       const int n = s_wch[e + 1] - s_wch[e];
       const int base = blocks / n, rem = blocks - base * n;
-      if (rem) atomicAdd(&s_len[len_class(base + 1)], rem);
-      atomicAdd(&s_len[len_class(base)], n - rem);
+      const int cl0 = len_class(base + 1), cl1 = len_class(base);
+      s_c[e] = rem;
+      s_c[E_tgt + e] = n - rem;
+      s_cl[e] = cl0;
+      s_cl[E_tgt + e] = cl1;
+      if (rem) atomicAdd(&s_len[cl0], rem);
+      atomicAdd(&s_len[cl1], n - rem);
     }
     __syncthreads();
-    if (tid == 0) {
-      int run = 0;
-      for (int l = WGRAD_LEN_BUCKETS; l >= 0; --l) {
-        const int c = s_len[l];
-        s_len[l] = run;
-        run += c;
+    if (warp == 0) {   // classes in descending order: lane p holds class BUCKETS - p; class 0 comes after all of them
+      static_assert(WGRAD_LEN_BUCKETS == 32, "one lane per non-zero length class");
+      const int v = s_len[WGRAD_LEN_BUCKETS - lane];
+      int incl = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
       }
+      s_start[WGRAD_LEN_BUCKETS - lane] = incl - v;
+      if (lane == 31) s_start[0] = incl;
     }
     __syncthreads();
     // within one class: experts in ascending order, an expert's longer chunks before its shorter ones.  One warp per
-    // class walks the experts 32 at a time.
-    for (int l = warp; l <= WGRAD_LEN_BUCKETS; l += PLAN_WARPS) {
-      int run = s_len[l];
+    // (non-empty) class walks the experts 32 at a time.
+    for (int l = warp; l <= WGRAD_LEN_BUCKETS; l += nwarps) {
+      if (s_len[l] == 0) continue;
+      int run = s_start[l];
       for (int e0 = 0; e0 < E_tgt; e0 += 32) {
         const int e = e0 + lane;
         int c0 = 0, c1 = 0;    // chunks of the expert's two lengths that fall into class l
         if (e < E_tgt) {
-          const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
-          const int n = s_wch[e + 1] - s_wch[e];
-          const int base = blocks / n, rem = blocks - base * n;
-          if (rem && len_class(base + 1) == l) c0 = rem;
-          if (len_class(base) == l) c1 = n - rem;
+          if (s_cl[e] == l) c0 = s_c[e];
+          if (s_cl[E_tgt + e] == l) c1 = s_c[E_tgt + e];
         }
         int incl = c0 + c1;
 #pragma unroll
@@ -276,7 +694,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
     }
     __syncthreads();
   }
-  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
+  for (int e = tid; e < E_tgt; e += nthr) {
     const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
     const int n = s_wch[e + 1] - s_wch[e];
     const int base = blocks / n, rem = blocks - base * n;
@@ -292,69 +710,104 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_kernel(const IdxT* __r
       pp.wchunk_rows[i] = rows;
     }
   }
-  // pad rows carry no slot
-  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
-    const int r0 = s_pad[e] + s_cnt[e], r1 = s_pad[e + 1];
-    for (int r = r0 + lane; r < r1; r += 32) pp.prow_to_slot[r] = -1;
-  }
 }
 
-template <typename IdxT>
-__global__ void __launch_bounds__(PLAN_THREADS) plan_permute_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
-                                                                    int R, int E_src, int E_tgt, int chunk, int nblk, PaddedPlan pp,
-                                                                    const int32_t* __restrict__ offsets, int32_t* __restrict__ row_to_slot,
-                                                                    int32_t* __restrict__ slot_to_row) {
-  extern __shared__ int32_t sm[];  // PLAN_WARPS*E + E ints
-  int32_t* s_shift = sm + PLAN_WARPS * E_tgt;
+
+__global__ void __launch_bounds__(PLAN_THREADS) plan_scan_kernel(int E_tgt, int nblk, PaddedPlan pp, int32_t* __restrict__ counts,
+                                                                 int32_t* __restrict__ offsets) {
+  extern __shared__ int32_t sm[];  // plan_scan_smem_ints(E_tgt) ints
+  __shared__ int s_warp_sum[PLAN_WARPS];
+  __shared__ int s_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
-  __syncthreads();
-  warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, pp.status);
-  __syncthreads();
-  // per-warp histogram -> first row of (block, warp, expert)
-  for (int e = tid; e < E_tgt; e += PLAN_THREADS) {
-    int base = offsets[e] + pp.blk_prefix[e * nblk + blockIdx.x];
+
+  // ---- this block's expert: exclusive prefix over blocks of its per-block counts, in place; the total is counts[e] ----
+  {
+    const int e = blockIdx.x;
+    int32_t* rowp = pp.blk_prefix + (size_t)e * nblk;
+    int carry = 0;
+    for (int b0 = 0; b0 < nblk; b0 += PLAN_THREADS * 8) {
+      const int b = b0 + tid * 8;
+      int v[8], sum = 0;
 #pragma unroll
-    for (int w = 0; w < PLAN_WARPS; ++w) {
-      const int t = sm[w * E_tgt + e];
-      sm[w * E_tgt + e] = base;
-      base += t;
+      for (int j = 0; j < 8; ++j) {
+        v[j] = (b + j < nblk) ? __ldcg(rowp + b + j) : 0;
+        sum += v[j];
+      }
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (lane == 31) s_warp_sum[warp] = incl;
+      __syncthreads();
+      int before = 0, total = 0;
+#pragma unroll
+      for (int w = 0; w < PLAN_WARPS; ++w) {
+        const int t = s_warp_sum[w];
+        if (w < warp) before += t;
+        total += t;
+      }
+      int run = carry + before + incl - sum;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (b + j < nblk) rowp[b + j] = run;
+        run += v[j];
+      }
+      carry += total;
+      __syncthreads();
     }
-    s_shift[e] = pp.row_shift[e];
+    if (tid == 0) counts[e] = carry;     // read back by the last block
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned t = atomicAdd(pp.ticket, 1u);
+    s_last = (t == (unsigned)(E_tgt - 1));
   }
   __syncthreads();
-  const int wlen = chunk / PLAN_WARPS;
-  const int base = blockIdx.x * chunk + warp * wlen;
-  int32_t* cur = sm + warp * E_tgt;
-  const unsigned lt = (1u << lane) - 1u;
-  const int key_bits = bits_for(E_tgt);
-  int raw_next = (base + lane < R) ? (int)idx[base + lane] : 0;   // ids are fetched one iteration ahead
-  for (int i = 0; i < wlen; i += 32) {
-    const int s = base + i + lane;
-    const bool valid = s < R;
-    const int raw = raw_next;
-    if (i + 32 < wlen && s + 32 < R) raw_next = (int)idx[s + 32];
-    const int e = valid ? fold_expert(raw, fold_map, E_src, E_tgt, pp.status) : -1;
-    const unsigned mask = same_key_lanes(e, key_bits);
-    const int row = valid ? cur[e] + __popc(mask & lt) : 0;
-    __syncwarp();
-    if (valid && lane == 31 - __clz(mask)) cur[e] = row + 1;
-    __syncwarp();
-    if (valid) {
-      const int prow = row + s_shift[e];
-      slot_to_row[s] = row;
-      row_to_slot[row] = s;
-      pp.slot_to_prow[s] = prow;
-      pp.prow_to_slot[prow] = s;
-    }
-    if (base + i + 32 >= R) break;
-  }
+  if (!s_last) return;
+  __threadfence();
+
+  for (int e = tid; e < E_tgt; e += PLAN_THREADS) sm[e] = __ldcg(counts + e);
+  plan_layout(sm, E_tgt, pp, counts, offsets);
 }
 
-// per-warp histograms while counting; the last block's scans and chunk ordering afterwards
-static int plan_hist_smem_ints(int E) {
-  const int a = PLAN_WARPS * E, b = 7 * E + 4 + WGRAD_LEN_BUCKETS + 2;
-  return a > b ? a : b;
+// ------------------------------------------------------------------------------------------------------------------
+// Launch
+// ------------------------------------------------------------------------------------------------------------------
+// Opt-in to more than 48 KB of dynamic shared memory: a per-device, per-kernel setting, raised when a launch needs more
+// than the kernel was last given on this device.  (The kernel is a template argument so that every kernel has its own
+// record: kernels with equal signatures share a function-pointer type.)
+template <auto Kern>
+static cudaError_t allow_smem(size_t bytes) {
+  static size_t granted[64] = {};
+  if (bytes <= 48 * 1024) return cudaSuccess;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (dev >= 0 && dev < 64 && granted[dev] >= bytes) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && dev >= 0 && dev < 64) granted[dev] = bytes;
+  return e;
+}
+
+template <typename IdxT, int V>
+static cudaError_t launch_counted(grouter_ctx* ctx, int phase, const IdxT* idx, const int32_t* fold_map, int32_t* offsets,
+                                  int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
+  const grouter_dims& dm = ctx->dims;
+  const int E = dm.E_tgt, nblk = ctx->geom.nblk;
+  if (phase == 0) {
+    const size_t sm0 = (size_t)PLAN_WARPS * E * 4 + (fold_map ? (size_t)dm.E_src * 2 : 0);
+    cudaError_t e = allow_smem<plan_count_kernel<IdxT, V>>(sm0);
+    if (e != cudaSuccess) return e;
+    plan_count_kernel<IdxT, V><<<nblk, PLAN_THREADS, sm0, st>>>(idx, fold_map, (int)ctx->R, dm.E_src, E, nblk, ctx->pp.blk_prefix, ctx->pp.status);
+  } else {
+    const size_t sm2 = (size_t)place_smem(dm.E_src, E, 16 * V, fold_map != nullptr).bytes;
+    cudaError_t e = allow_smem<plan_place_kernel<IdxT, V>>(sm2);
+    if (e != cudaSuccess) return e;
+    plan_place_kernel<IdxT, V><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, (int)ctx->R, dm.E_src, E, nblk, ctx->pp, offsets, row_to_slot, slot_to_row);
+  }
+  return cudaGetLastError();
 }
 
 template <typename IdxT>
@@ -363,18 +816,28 @@ static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, c
   const grouter_dims& dm = ctx->dims;
   const int R = (int)ctx->R, E = dm.E_tgt;
   const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
+  if (phase == 1) {
+    const size_t sm1 = sizeof(int32_t) * (size_t)plan_scan_smem_ints(E);
+    plan_scan_kernel<<<E, PLAN_THREADS, sm1, st>>>(E, nblk, ctx->pp, counts, offsets);
+    return cudaGetLastError();
+  }
+  switch (ctx->geom.ipt) {
+    case 16: return launch_counted<IdxT, 1>(ctx, phase, idx, fold_map, offsets, row_to_slot, slot_to_row, st);
+    case 32: return launch_counted<IdxT, 2>(ctx, phase, idx, fold_map, offsets, row_to_slot, slot_to_row, st);
+    case 64: return launch_counted<IdxT, 4>(ctx, phase, idx, fold_map, offsets, row_to_slot, slot_to_row, st);
+    default: break;
+  }
   if (phase == 0) {
-    const size_t sm1 = sizeof(int32_t) * (size_t)plan_hist_smem_ints(E);
-    plan_hist_kernel<IdxT><<<nblk, PLAN_THREADS, sm1, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, counts, offsets);
+    const size_t sm0 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E);
+    plan_hist_ballot_kernel<IdxT><<<nblk, PLAN_THREADS, sm0, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp.blk_prefix, ctx->pp.status);
   } else {
-    const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + E);
-    plan_permute_kernel<IdxT><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, offsets,
-                                                               row_to_slot, slot_to_row);
+    const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + 2 * (E + 1));
+    plan_permute_ballot_kernel<IdxT><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, offsets,
+                                                                      row_to_slot, slot_to_row);
   }
   return cudaGetLastError();
 }
 
-// phase 0: histogram + scans (counts, offsets, padded layout); phase 1: stable permutation.
 cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int32_t* fold_map, int32_t* counts, int32_t* offsets,
                         int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
   if (ctx->dims.idx_dtype == GROUTER_IDX_U8)
@@ -385,10 +848,10 @@ cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int3
 }  // namespace grouter
 
 // ------------------------------------------------------------------------
-// grouter_plan_noalloc: the same two plan kernels, run without a context.
+// grouter_plan_noalloc: the same plan kernels, run without a context.
 //
 // grouter_create owns the plan's scratch (per-block histograms, the ticket of
-// the last-block scan, the padded copy of the permutation) in memory it gets
+// the last-block scan, the padded layout and the work lists) in memory it gets
 // from cudaMalloc.  Some hosts cannot make that call: a process that has
 // handed the whole device to a pooling allocator with a fixed reservation, a
 // plug-in running under a memory budget it may not exceed, or a
@@ -404,12 +867,14 @@ namespace {
 constexpr int NOALLOC_MAX_R = 1 << 19;       // routed slots T*k
 constexpr int NOALLOC_MAX_E = 256;           // target experts
 constexpr int NOALLOC_MAX_ROWS = NOALLOC_MAX_R + ROW_TILE * NOALLOC_MAX_E;          // padded rows
-constexpr int NOALLOC_MAX_BLOCKS = NOALLOC_MAX_R / PLAN_MIN_CHUNK;                   // plan_geom never uses more
+constexpr int NOALLOC_MAX_BLOCKS = NOALLOC_MAX_R / PLAN_MIN_CHUNK;                   // plan_geom never uses more (either form)
+static_assert(16 * PLAN_THREADS >= PLAN_MIN_CHUNK, "the counted form's smallest chunk must not be shorter than the ballot form's");
 // layout of the scratch, in 32-bit words (every part starts on a 256-byte boundary)
 constexpr int NA_PAD_OFFSETS = 0;                                     // [E+1]
 constexpr int NA_ROW_SHIFT = NA_PAD_OFFSETS + 320;                    // [E]
 constexpr int NA_PAD_BEGIN = NA_ROW_SHIFT + 256;                      // [E]
-constexpr int NA_N_TILES = NA_PAD_BEGIN + 256;                        // [1]
+constexpr int NA_PAIR_PREFIX = NA_PAD_BEGIN + 256;                    // [E+1]
+constexpr int NA_N_TILES = NA_PAIR_PREFIX + 320;                      // [1]
 constexpr int NA_TICKET = NA_N_TILES + 64;                            // [1]
 constexpr int NA_STATUS = NA_TICKET + 64;                             // [1] used when the caller passes no status word
 constexpr int NA_PAIR_ROW0 = NA_STATUS + 64;                          // [rows/128]
@@ -419,14 +884,12 @@ constexpr int NA_WCHUNK_EXPERT = NA_PAIR_EXPERT + NOALLOC_MAX_ROWS / ROW_TILE; /
 constexpr int NA_WCHUNK_ROW0 = NA_WCHUNK_EXPERT + NOALLOC_MAX_WCHUNKS;         // [chunks]
 constexpr int NA_WCHUNK_ROWS = NA_WCHUNK_ROW0 + NOALLOC_MAX_WCHUNKS;           // [chunks]
 constexpr int NA_N_WCHUNKS = NA_WCHUNK_ROWS + NOALLOC_MAX_WCHUNKS;             // [1]
-constexpr int NA_SLOT_TO_PROW = NA_N_WCHUNKS + 64;                             // [R]
-constexpr int NA_PROW_TO_SLOT = NA_SLOT_TO_PROW + NOALLOC_MAX_R;      // [rows]
-constexpr int NA_BLK_PREFIX = NA_PROW_TO_SLOT + NOALLOC_MAX_ROWS;     // [E * blocks]
+constexpr int NA_BLK_PREFIX = NA_N_WCHUNKS + 64;                      // [E * blocks]
 constexpr int NA_WORDS = NA_BLK_PREFIX + NOALLOC_MAX_E * NOALLOC_MAX_BLOCKS;
-static_assert(NA_PAIR_ROW0 % 64 == 0 && NA_PAIR_EXPERT % 64 == 0 && NA_SLOT_TO_PROW % 64 == 0 && NA_PROW_TO_SLOT % 64 == 0 && NA_BLK_PREFIX % 64 == 0,
+static_assert(NA_PAIR_ROW0 % 64 == 0 && NA_PAIR_EXPERT % 64 == 0 && NA_WCHUNK_EXPERT % 64 == 0 && NA_BLK_PREFIX % 64 == 0,
               "scratch parts must start on 256-byte boundaries");
 
-// About 4.6 MB per GPU.  In host code this name is only a handle for cudaGetSymbolAddress: it is not a
+// About 0.3 MB per GPU.  In host code this name is only a handle for cudaGetSymbolAddress: it is not a
 // device address and must never be handed to a kernel as one.
 static __device__ __align__(256) int32_t g_plan_scratch[NA_WORDS];
 
@@ -476,14 +939,15 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   int32_t* base = plan_scratch_on_current_device(&rc);
   if (!base) return rc;
 
-  grouter_ctx c{};   // lives on the host stack for the duration of the two launches
+  grouter_ctx c{};   // lives on the host stack for the duration of the launches
   c.dims.T = T; c.dims.d = 8; c.dims.ffn = 8; c.dims.E_src = E_src; c.dims.E_tgt = E_tgt; c.dims.k = k;
   c.dims.idx_dtype = idx_dtype; c.dims.gate_dtype = GROUTER_GATE_BF16;
   c.R = (int64_t)T * k;
-  c.geom = plan_geom(c.R);
+  c.geom = plan_geom(c.R, E_src, E_tgt);
   c.pp.pad_offsets = base + NA_PAD_OFFSETS;
   c.pp.row_shift = base + NA_ROW_SHIFT;
   c.pp.pad_begin = base + NA_PAD_BEGIN;
+  c.pp.pair_prefix = base + NA_PAIR_PREFIX;
   c.pp.n_pair_tiles = base + NA_N_TILES;
   c.pp.ticket = reinterpret_cast<unsigned int*>(base + NA_TICKET);
   c.pp.tile_counter = c.pp.ticket + 4;
@@ -495,8 +959,6 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.pp.wchunk_row0 = base + NA_WCHUNK_ROW0;
   c.pp.wchunk_rows = base + NA_WCHUNK_ROWS;
   c.pp.n_wchunks = base + NA_N_WCHUNKS;
-  c.pp.slot_to_prow = base + NA_SLOT_TO_PROW;
-  c.pp.prow_to_slot = base + NA_PROW_TO_SLOT;
   c.pp.blk_prefix = base + NA_BLK_PREFIX;
   if (c.geom.nblk > NOALLOC_MAX_BLOCKS) return GROUTER_ERR_UNSUPPORTED;
 
@@ -505,7 +967,7 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   // word must start clear; every other part is overwritten before it is read.
   if (cudaMemsetAsync(c.pp.ticket, 0, sizeof(unsigned int), st) != cudaSuccess) return GROUTER_ERR_CUDA;
   if (cudaMemsetAsync(c.pp.status, 0, sizeof(int32_t), st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  for (int phase = 0; phase < 2; ++phase)
+  for (int phase = 0; phase < PLAN_PHASES; ++phase)
     if (launch_plan(&c, phase, idx, fold_map, counts, offsets, row_to_slot, slot_to_row, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   return GROUTER_OK;
 }
