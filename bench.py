@@ -197,6 +197,35 @@ def routing_stats_leg(dev, idx, E, seq_len=4096, n_nodes=8, iters=20):
             "algorithmic_bytes": by, "gbs": by / (ms * 1e-3) / 1e9, "max_vio": float(mv.item())}
 
 
+def combine_ab_leg(dev, w, layer, idx, fm, gates, X, W_gu, W_d, rounds=5, per_round=3):
+    """Forward pass with the combine as its own kernel against the combine folded into the down product's epilogue
+    (GROUTER_FLAG_FUSED_COMBINE), interleaved in one process so that both see the same clocks."""
+    import torch
+    from paper_2603_06626_b200 import binding
+    fused = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt, device=str(dev), flags=binding.FLAG_FUSED_COMBINE)
+    Y = torch.empty_like(X)
+    layer.plan(idx, fm)
+    fused.plan(idx, fm)
+    times = {"separate": [], "fused": []}
+    for name, ly in (("separate", layer), ("fused", fused)):     # warm-up
+        ly.forward(X, gates, W_gu, W_d, Y)
+    torch.cuda.synchronize()
+    for _ in range(rounds):
+        for name, ly in (("separate", layer), ("fused", fused)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(per_round):
+                ly.forward(X, gates, W_gu, W_d, Y)
+            e1.record()
+            torch.cuda.synchronize()
+            times[name].append(e0.elapsed_time(e1) / per_round)
+    fused.check_status()
+    fused.close()
+    med = {k: statistics.median(v) for k, v in times.items()}
+    return {"forward_ms_separate_combine": med["separate"], "forward_ms_fused_combine": med["fused"],
+            "fused_over_separate": med["fused"] / med["separate"], "rounds": rounds, "forwards_per_round": per_round}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -612,6 +641,8 @@ def main():
     }
     if e2e is not None:
         line["e2e"] = e2e
+    if world == 1 and not args.no_isolated:
+        line["combine_ab"] = combine_ab_leg(dev, w, layer, idx, fm, gates, X, W_gu, W_d)
     if world == 1 and not args.no_plan_scale:
         layer.close()
         torch.cuda.synchronize()

@@ -57,7 +57,12 @@ enum { GROUTER_IDX_U8 = 0, GROUTER_IDX_I32 = 1 };
 enum { GROUTER_GATE_BF16 = 0, GROUTER_GATE_F32 = 1 };
 /* grouter_moe_bwd adds the weight gradients into dW_gu / dW_d instead of overwriting them (gradient accumulation
  * over micro-batches; the caller zeroes them before the first one).  Experts without slots are left untouched. */
-enum { GROUTER_FLAG_ACCUMULATE_DW = 1 };
+enum { GROUTER_FLAG_ACCUMULATE_DW = 1,
+       /* grouter_moe_fwd folds the combine of Eq. 1 into the down product: its epilogue adds every gate-weighted routed row
+        * into an fp32 [T, d] accumulator in the workspace (16-byte reductions) and one more pass rounds it to bf16 Y; the
+        * expert-ordered output rows are never written.  The order of a token's k additions is not fixed, so Y may differ
+        * in its last bits from run to run (without the flag it is bit-reproducible).  The workspace grows by 4*T*d bytes. */
+       GROUTER_FLAG_FUSED_COMBINE = 2 };
 
 typedef struct grouter_ctx grouter_ctx; /* opaque */
 
@@ -237,6 +242,19 @@ int grouter_host_wait(grouter_ctx* ctx, int32_t steps_in_flight);
 int grouter_status(grouter_ctx* ctx, void* stream);
 
 const char* grouter_strerror(int code);
+
+/* Every device-side wait of this library's kernels (an operand stage, an accumulator, the next tile number) gives up
+ * after a limit, 4 s by default; the CTA then sets GROUTER_ERR_TIMEOUT in the status word, waits for its own copies in
+ * flight, frees its tensor memory and returns, so the context stays usable.  grouter_set_wait_limit changes the limit
+ * for this context's later launches (1 .. 60,000,000 us).  The paper has no counterpart: failure handling of this
+ * implementation. */
+int grouter_set_wait_limit(grouter_ctx* ctx, int64_t microseconds);
+/* Self-test of that mechanism without disturbing a pipeline: launches one thread that waits, with the same bounded
+ * wait the GEMMs use, on a barrier nothing ever arrives at, for limit_microseconds (1 .. 1,000,000).  The wait runs
+ * out, the kernel sets the timeout bit in the context's status word and returns; the call synchronises `stream` and
+ * writes how long the kernel waited to *waited_microseconds (host).  grouter_status then reports
+ * GROUTER_ERR_TIMEOUT once and clears it. */
+int grouter_wait_selftest(grouter_ctx* ctx, int64_t limit_microseconds, int64_t* waited_microseconds, void* stream);
 
 /* Per-kernel device timing (measurement aid; no counterpart in the paper).
  * grouter_timing_enable(ctx, n) creates n CUDA event pairs (host call, allocates;

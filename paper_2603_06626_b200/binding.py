@@ -16,13 +16,14 @@ from . import build as _build
 
 IDX_U8, IDX_I32 = 0, 1
 FLAG_ACCUMULATE_DW = 1
+FLAG_FUSED_COMBINE = 2
 NORM_SOFTMAX, NORM_SIGMOID = 0, 1
 GATE_BF16, GATE_F32 = 0, 1
 
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
-           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read"]
+           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW", "plan_scan"]
 
@@ -94,6 +95,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_gemm_cycles_read.restype = ctypes.c_int
     lib.grouter_wgrad_chunk_rows.argtypes = [vp]
     lib.grouter_wgrad_chunk_rows.restype = ctypes.c_int32
+    lib.grouter_set_wait_limit.argtypes = [vp, ctypes.c_int64]
+    lib.grouter_set_wait_limit.restype = ctypes.c_int
+    lib.grouter_wait_selftest.argtypes = [vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64), vp]
+    lib.grouter_wait_selftest.restype = ctypes.c_int
     lib.grouter_timing_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.grouter_timing_read.restype = ctypes.c_int
     if path == _build.LIB:
@@ -219,6 +224,17 @@ class GrouterLayer:
         names = ["gemm_up_swiglu", "gemm_down", "gemm_dH", "gemm_dX", "wgrad_down", "wgrad_gate_up"]
         keys = ["cycles", "wait_operands", "wait_accumulator", "tiles", "k_steps"]
         return {n: {k: int(buf[5 * i + j]) for j, k in enumerate(keys)} for i, n in enumerate(names)}
+
+    def set_wait_limit(self, microseconds: int) -> None:
+        """Limit of every bounded device-side wait of this context's later launches."""
+        _check(self.lib.grouter_set_wait_limit(self.ctx, microseconds), "grouter_set_wait_limit")
+
+    def wait_selftest(self, limit_microseconds: int) -> int:
+        """One bounded wait that cannot succeed; returns the microseconds the kernel waited.  Leaves GROUTER_ERR_TIMEOUT in
+        the status word (read and cleared by status())."""
+        waited = ctypes.c_int64(0)
+        _check(self.lib.grouter_wait_selftest(self.ctx, limit_microseconds, ctypes.byref(waited), _stream()), "grouter_wait_selftest")
+        return int(waited.value)
 
     def timing_read(self):
         """-> {kernel name: (total ms, launches)} since the last read; synchronises the current stream."""

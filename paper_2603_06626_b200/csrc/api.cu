@@ -16,7 +16,7 @@ int check_dims(const grouter_dims* dm) {
   if (dm->T < 1 || dm->d < 1 || dm->ffn < 1 || dm->E_src < 1 || dm->E_tgt < 1 || dm->k < 1) return GROUTER_ERR_INVALID_ARG;
   if (dm->idx_dtype != GROUTER_IDX_U8 && dm->idx_dtype != GROUTER_IDX_I32) return GROUTER_ERR_INVALID_ARG;
   if (dm->gate_dtype != GROUTER_GATE_BF16 && dm->gate_dtype != GROUTER_GATE_F32) return GROUTER_ERR_INVALID_ARG;
-  if (dm->flags & ~GROUTER_FLAG_ACCUMULATE_DW) return GROUTER_ERR_INVALID_ARG;
+  if (dm->flags & ~(GROUTER_FLAG_ACCUMULATE_DW | GROUTER_FLAG_FUSED_COMBINE)) return GROUTER_ERR_INVALID_ARG;
   if (dm->d % 8 || dm->ffn % 8) return GROUTER_ERR_UNSUPPORTED;
   if (dm->E_tgt > 1024 || dm->k > 32) return GROUTER_ERR_UNSUPPORTED;
   if (dm->idx_dtype == GROUTER_IDX_U8 && dm->E_src > 256) return GROUTER_ERR_UNSUPPORTED;
@@ -97,6 +97,7 @@ Workspace carve_workspace(const grouter_dims& dm, int64_t Rp, void* base) {
   const size_t rd = (size_t)Rp * dm.d * 2, rf = (size_t)Rp * dm.ffn * 2;
   const size_t oXp = take(rd), oG = take(rf), oU = take(rf), oH = take(rf), oO = take(rd), odY = take(rd), odGU = take(2 * rf);
   const size_t oPart = take((size_t)(2 * ((dm.ffn + 255) / 256)) * Rp * 4);
+  const size_t oYacc = take((dm.flags & GROUTER_FLAG_FUSED_COMBINE) ? (size_t)dm.T * dm.d * 4 : 0);
   w.bytes = off;
   if (b) {
     w.Xp = reinterpret_cast<__nv_bfloat16*>(b + oXp);
@@ -107,6 +108,7 @@ Workspace carve_workspace(const grouter_dims& dm, int64_t Rp, void* base) {
     w.dYp = reinterpret_cast<__nv_bfloat16*>(b + odY);
     w.dGU = reinterpret_cast<__nv_bfloat16*>(b + odGU);
     w.dgate_part = reinterpret_cast<float*>(b + oPart);
+    w.Yacc = (dm.flags & GROUTER_FLAG_FUSED_COMBINE) ? reinterpret_cast<float*>(b + oYacc) : nullptr;
   }
   return w;
 }
@@ -177,6 +179,8 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->idle_gap_us = 0;
   c->count_cycles = false;
   c->d_cycles = nullptr;
+  c->wait_limit_ns = DEFAULT_WAIT_LIMIT_NS;
+  c->d_waited = nullptr;
   c->s_in = c->s_out = nullptr;
   for (int i = 0; i < 2; ++i) c->ev_in_fwd[i] = c->ev_in_bwd[i] = c->ev_fwd_done[i] = c->ev_bwd_done[i] = c->ev_out_done[i] = nullptr;
   {
@@ -200,7 +204,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   const size_t o_pr = take((size_t)c->max_m_tiles * 4), o_pe = take((size_t)c->max_m_tiles * 4), o_nt = take(4);
   const size_t o_we = take((size_t)c->max_wchunks * 4), o_wr = take((size_t)c->max_wchunks * 4), o_wn = take((size_t)c->max_wchunks * 4), o_nw = take(4);
   const size_t o_bp = take((size_t)E * c->geom.nblk * 4), o_tk = take(4), o_st = take(4);
-  const size_t o_cy = take(6 * GEMM_CYCLE_COUNTERS * sizeof(unsigned long long));
+  const size_t o_cy = take(6 * GEMM_CYCLE_COUNTERS * sizeof(unsigned long long)), o_wt = take(sizeof(unsigned long long));
   if (cudaMalloc(&c->d_block, off) != cudaSuccess) {
     c->d_block = nullptr;
     grouter_destroy(c);
@@ -227,6 +231,7 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.tile_counter = c->pp.ticket + 4;   // same 256-byte slot
   c->pp.status = reinterpret_cast<int32_t*>(b + o_st);
   c->d_cycles = reinterpret_cast<unsigned long long*>(b + o_cy);
+  c->d_waited = reinterpret_cast<unsigned long long*>(b + o_wt);
   *out = c;
   return GROUTER_OK;
 }
@@ -284,13 +289,30 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
     Timed tm(ctx, 3, st);
     if (launch_grouped_gemm(ctx, MODE_UP, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
-  {
-    Timed tm(ctx, 4, st);
-    if (launch_grouped_gemm(ctx, MODE_DOWN, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-  }
-  {
-    Timed tm(ctx, 5, st);
-    if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (ctx->dims.flags & GROUTER_FLAG_FUSED_COMBINE) {
+    // the down product adds every routed row into the token's fp32 row; a last pass rounds to bf16
+    const size_t n = (size_t)ctx->dims.T * ctx->dims.d;
+    {
+      Timed tm(ctx, 5, st);
+      if (cudaMemsetAsync(ws.Yacc, 0, n * sizeof(float), st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    }
+    {
+      Timed tm(ctx, 4, st);
+      if (launch_grouped_gemm(ctx, MODE_DOWN_ADD, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    }
+    {
+      Timed tm(ctx, 5, st);
+      if (launch_cast_rows(ctx, ws.Yacc, static_cast<__nv_bfloat16*>(Y), n, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    }
+  } else {
+    {
+      Timed tm(ctx, 4, st);
+      if (launch_grouped_gemm(ctx, MODE_DOWN, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    }
+    {
+      Timed tm(ctx, 5, st);
+      if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+    }
   }
   ctx->forwarded = true;
   return GROUTER_OK;
@@ -407,7 +429,11 @@ int grouter_status(grouter_ctx* ctx, void* stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return GROUTER_ERR_CUDA;
   if (h != 0) {
     if (cudaMemsetAsync(ctx->pp.status, 0, 4, st) != cudaSuccess) return GROUTER_ERR_CUDA;
-    if (h & STATUS_TIMEOUT) return GROUTER_ERR_TIMEOUT;
+    if (h & STATUS_TIMEOUT) {
+      // a grouped GEMM that gave up left its tile counter mid-count: the next launch must start from zero again
+      if (cudaMemsetAsync(ctx->pp.tile_counter, 0, sizeof(unsigned int), st) != cudaSuccess) return GROUTER_ERR_CUDA;
+      return GROUTER_ERR_TIMEOUT;
+    }
     return GROUTER_ERR_BAD_INDEX;
   }
   return GROUTER_OK;
@@ -469,6 +495,23 @@ int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t
     launches[ctx->ev_slot[i]] += 1;
   }
   ctx->ev_used = 0;
+  return GROUTER_OK;
+}
+
+int grouter_set_wait_limit(grouter_ctx* ctx, int64_t microseconds) {
+  if (!ctx || microseconds < 1 || microseconds > 60000000) return GROUTER_ERR_INVALID_ARG;
+  ctx->wait_limit_ns = (unsigned long long)microseconds * 1000ull;
+  return GROUTER_OK;
+}
+
+int grouter_wait_selftest(grouter_ctx* ctx, int64_t limit_microseconds, int64_t* waited_microseconds, void* stream) {
+  if (!ctx || !waited_microseconds || limit_microseconds < 1 || limit_microseconds > 1000000) return GROUTER_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (launch_wait_selftest(ctx, (unsigned long long)limit_microseconds * 1000ull, ctx->d_waited, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  unsigned long long ns = 0;
+  if (cudaMemcpyAsync(&ns, ctx->d_waited, sizeof(ns), cudaMemcpyDeviceToHost, st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return GROUTER_ERR_CUDA;
+  *waited_microseconds = (int64_t)(ns / 1000ull);
   return GROUTER_OK;
 }
 

@@ -12,6 +12,7 @@ namespace grouter {
 // Sticky device status bits (ORed into ctx->d_status).
 constexpr int STATUS_BAD_INDEX = 1;
 constexpr int STATUS_TIMEOUT = 2;
+constexpr unsigned long long DEFAULT_WAIT_LIMIT_NS = 4000000000ull;   // bounded device-side waits give up after this long
 
 constexpr int ROW_TILE = 128;        // rows one CTA owns in a GEMM tile; expert segments are padded to it
 constexpr int PAIR_VALID2 = 1 << 30; // flag in PaddedPlan::pair_expert
@@ -114,6 +115,8 @@ struct grouter_ctx {
   int idle_gap_us;        // measurement aid: idle time inserted after every timed kernel (0 = none)
   bool count_cycles;      // measurement aid: the grouped GEMMs account for their issuers' cycles
   unsigned long long* d_cycles;   // device [6 GEMMs][GEMM_CYCLE_COUNTERS], summed over CTA pairs and launches
+  unsigned long long wait_limit_ns;   // limit of every bounded device-side wait of this context's kernels
+  unsigned long long* d_waited;   // device [1] scratch of grouter_wait_selftest
 };
 
 namespace grouter {
@@ -128,6 +131,7 @@ struct Workspace {
   __nv_bfloat16* dYp;   // [R_pad_max, d]   gathered upstream gradient
   __nv_bfloat16* dGU;   // [R_pad_max, 2F]  [dG | dU]
   float* dgate_part;    // [2*ceil(F/256), R_pad_max] partial row sums for d-gate
+  float* Yacc;          // [T, d] fp32 sum of the routed rows (only with GROUTER_FLAG_FUSED_COMBINE)
   size_t bytes;
 };
 Workspace carve_workspace(const grouter_dims& dm, int64_t R_pad_max, void* base);
@@ -142,10 +146,13 @@ cudaError_t launch_plan(grouter_ctx* ctx, int phase, const void* idx, const int3
 cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st);
 // out[t,:] = sum_j src[prow(t*k+j),:] (fp32 sum in slot order); optionally
 // dgates[t,j] = sum_n dgate_part[n][prow].
+// out[i] = bf16(in[i]) for n elements (n a multiple of 8).
+cudaError_t launch_cast_rows(grouter_ctx* ctx, const float* in, __nv_bfloat16* out, size_t n, cudaStream_t st);
 cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part,
                                int n_part, float* dgates, cudaStream_t st);
 
-enum GemmMode { MODE_UP = 0, MODE_DOWN = 1, MODE_DH = 2, MODE_DX = 3, MODE_WGRAD_D = 4, MODE_WGRAD_GU = 5, MODE_DENSE = 6 };
+// MODE_DOWN_ADD: the down product with the combine folded into its epilogue (fp32 reductions into a [T, d] accumulator).
+enum GemmMode { MODE_UP = 0, MODE_DOWN = 1, MODE_DH = 2, MODE_DX = 3, MODE_WGRAD_D = 4, MODE_WGRAD_GU = 5, MODE_DENSE = 6, MODE_DOWN_ADD = 7 };
 
 cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace& ws, const void* gates, const void* W_gu,
                                 const void* W_d, float* dW_gu, float* dW_d, cudaStream_t st);
@@ -153,6 +160,8 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
 cudaError_t launch_zero_split_dw(grouter_ctx* ctx, float* dW_gu, float* dW_d, cudaStream_t st);
 // A kernel that only lets `microseconds` pass (one thread watching the global timer, capped at one second).
 cudaError_t launch_idle(int microseconds, cudaStream_t st);
+// Measures one bounded wait that cannot succeed (see grouter_wait_selftest).
+cudaError_t launch_wait_selftest(grouter_ctx* ctx, unsigned long long limit_ns, unsigned long long* d_waited_ns, cudaStream_t st);
 cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,
                               cudaStream_t st);
 

@@ -58,7 +58,7 @@ struct GemmParams {
   const int32_t* wchunk_expert;// device [chunks] expert | WCHUNK_SPLIT
   const int32_t* wchunk_row0;  // device [chunks] first padded row
   const int32_t* wchunk_rows;  // device [chunks] rows, multiple of 64
-  int32_t E, d, F;
+  int32_t E, d, F, k;
   int32_t accumulate;          // weight-gradient modes: add every tile into the caller's gradient
   int32_t M, N, K;             // DENSE: problem; WGRAD: per-expert output M x N
   int32_t tiles_m, tiles_n;    // output tiles per problem (tiles_m unused by row-parallel modes)
@@ -71,10 +71,11 @@ struct GemmParams {
   int32_t gate_is_f32;
   const __nv_bfloat16* in_G;   // DH
   const __nv_bfloat16* in_U;   // DH
-  float* out_f;                // DH: dgate_part; weight gradients / DENSE: the fp32 output [E, M, N]
+  float* out_f;                // DH: dgate_part; weight gradients / DENSE: the fp32 output [E, M, N]; DOWN_ADD: Y accumulator [T, d]
   int32_t* status;
   unsigned int* tile_counter;  // device scalar, zero at launch (unused by DENSE, which has no context to keep one)
   unsigned long long* cycles;  // null, or GEMM_CYCLE_COUNTERS counters every issuer adds its account to
+  unsigned long long wait_limit_ns;   // how long any one wait (barrier, tile queue) may last before the CTA gives up
 };
 
 struct Tile {     // one CTA's share of a pair tile
@@ -100,7 +101,7 @@ template <int MODE>
 __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank) {
   Tile ti;
   ti.add = false;
-  if (MODE == MODE_UP || MODE == MODE_DOWN || MODE == MODE_DH || MODE == MODE_DX) {
+  if (MODE == MODE_UP || MODE == MODE_DOWN || MODE == MODE_DOWN_ADD || MODE == MODE_DH || MODE == MODE_DX) {
     const int mt = t / p.tiles_n, nt = t - mt * p.tiles_n;
     const int pe = __ldg(p.pair_expert + mt);
     ti.e = pe & ~PAIR_VALID2;
@@ -116,7 +117,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
       ti.b_x = 0;
       ti.b_y = ti.e * 2 * p.F + rank * p.F + ti.col0;
       ti.num_k = (p.d + BK - 1) / BK;
-    } else if (MODE == MODE_DOWN) { // B = W_d as [E*d, F], K-major
+    } else if (MODE == MODE_DOWN || MODE == MODE_DOWN_ADD) { // B = W_d as [E*d, F], K-major
       ti.col0 = nt * BN;
       ti.n_valid = min(BN, p.d - ti.col0);
       ti.b_x = 0;
@@ -297,7 +298,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (seq == want) return (int)v;
       }
       if (*abort_flag) return 0x7fffffff;
-      if (ptx::globaltimer_ns() - t0 > 4000000000ull) {
+      if (ptx::globaltimer_ns() - t0 > p.wait_limit_ns) {
         *abort_flag = 1;
         return 0x7fffffff;
       }
@@ -338,7 +339,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const Tile ti = decode_tile<MODE>(p, t, rank);
         bool ok = true;
         for (int ks = 0; ks < ti.steps; ++ks) {
-          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) {
+          if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.wait_limit_ns)) {
             ok = false;
             break;
           }
@@ -379,7 +380,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       // every stage release the leader has multicast to this CTA must have landed before the CTA may exit
       for (int i = 0; i < STAGES && !*abort_flag; ++i) {
-        if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag)) break;
+        if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, p.wait_limit_ns)) break;
         if (++s == STAGES) {
           s = 0;
           ph ^= 1u;
@@ -413,7 +414,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int t = DYN ? next_tile() : pair_id; t < n_tiles && !*abort_flag; t = DYN ? next_tile() : t + n_pairs) {
         const Tile ti = decode_tile<MODE>(p, t, 0);
         const long long c_t0 = count ? clock64() : 0;
-        if (!ptx::mbar_wait_bounded(tempty_bar(acc), acc_ph ^ 1u, abort_flag)) break;
+        if (!ptx::mbar_wait_bounded(tempty_bar(acc), acc_ph ^ 1u, abort_flag, p.wait_limit_ns)) break;
         if (count) {
           c_acc += clock64() - c_t0;
           n_tiles_done += 1;
@@ -424,7 +425,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         bool ok = true;
         for (int ks = 0; ks < ti.steps; ++ks) {
           const long long c_k0 = count ? clock64() : 0;
-          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag)) {
+          if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, p.wait_limit_ns)) {
             ok = false;
             break;
           }
@@ -523,7 +524,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const bool live = ti.m_valid > 0;    // false: this CTA only lent its half of B to the pair
       uint4 g4[4], u4[4];
       if (MODE == MODE_DH) load_gu(ti, 0, g4, u4);   // in flight while the main loop of this tile finishes
-      if (!ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag)) break;
+      if (!ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag, p.wait_limit_ns)) break;
       ptx::tc_fence_after();
       const uint32_t t_row = tmem_base + (uint32_t)acc * BN + ((uint32_t)(quad * 32) << 16);
       const bool have_acc = ti.num_k > 0;
@@ -585,6 +586,30 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               stage_put_bf16(sb, cc * 4, v);
             }
             stage_send_2d(sb, &tmC0, ti.col0 + cb, y0);
+          }
+        }
+      } else if (MODE == MODE_DOWN_ADD) {
+        // Combine folded into the product (Eq. 1): this thread's row belongs to one token; its gate-weighted expert
+        // output is added to the token's fp32 row with 16-byte reductions.  The order in which a token's k rows arrive
+        // is not fixed, so Y may differ in the last bits from run to run.
+        int tok = -1;
+        if (live) {
+          const int prow = ti.row0 + r;
+          if (prow < __ldg(p.pad_begin + ti.e)) tok = __ldg(p.row_to_slot + (prow - __ldg(p.row_shift + ti.e))) / p.k;
+        }
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c0 = half * 128 + cc * 32;
+          if (live && ti.n_valid - c0 > 0) {             // warp-uniform
+            uint32_t ra[32];
+            ptx::tmem_ld32(t_row + c0, ra);
+            ptx::tmem_ld_wait();
+            if (tok >= 0) {
+              float* dst = p.out_f + (size_t)tok * p.d + ti.col0 + c0;
+#pragma unroll
+              for (int q = 0; q < 8; ++q)
+                if (c0 + 4 * q < ti.n_valid) ptx::red_add_v4_f32(dst + 4 * q, ra[4 * q], ra[4 * q + 1], ra[4 * q + 2], ra[4 * q + 3]);
+            }
           }
         }
       } else if (MODE == MODE_DH) {
@@ -786,6 +811,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.E = E;
   p.d = d;
   p.F = F;
+  p.k = dm.k;
   p.R_pad_max = ctx->R_pad_max;
   p.accumulate = (dm.flags & GROUTER_FLAG_ACCUMULATE_DW) ? 1 : 0;
   p.row_to_slot = ctx->pp.row_to_slot;
@@ -795,7 +821,8 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.gate_is_f32 = dm.gate_dtype == GROUTER_GATE_F32;
   p.status = ctx->pp.status;
   p.tile_counter = ctx->pp.tile_counter;
-  p.cycles = ctx->count_cycles ? ctx->d_cycles + (int)mode * GEMM_CYCLE_COUNTERS : nullptr;
+  p.cycles = ctx->count_cycles ? ctx->d_cycles + (int)(mode == MODE_DOWN_ADD ? MODE_DOWN : mode) * GEMM_CYCLE_COUNTERS : nullptr;
+  p.wait_limit_ns = ctx->wait_limit_ns;
   Maps m;
   bool ok = true;
   const int grid = ctx->num_sms & ~1;   // whole CTA pairs, one CTA per SM
@@ -812,6 +839,13 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
       p.tiles_n = cdiv(d, BN);
       if (!ok) return cudaErrorInvalidValue;
       return launch_t<MODE_DOWN, false, false>(m, p, grid, st);
+    case MODE_DOWN_ADD:
+      ok = make_map(&m.A, ws.Hs, Rp, F, 128) && make_map(&m.B, W_d, (uint64_t)E * d, F, 128);
+      m.C0 = m.C1 = m.C2 = m.A;   // results leave as reductions, without a tensor map
+      p.tiles_n = cdiv(d, BN);
+      p.out_f = ws.Yacc;
+      if (!ok) return cudaErrorInvalidValue;
+      return launch_t<MODE_DOWN_ADD, false, false>(m, p, grid, st);
     case MODE_DH:
       // [dG|dU] is one [R_pad, 2F] buffer; the stores see it as two [R_pad, F] views so that clipping stops at F
       ok = make_map(&m.A, ws.dYp, Rp, d, 128) && make_map(&m.B, W_d, (uint64_t)E * d, F, 64) &&
@@ -874,6 +908,27 @@ cudaError_t launch_zero_split_dw(grouter_ctx* ctx, float* dW_gu, float* dW_d, cu
   return cudaGetLastError();
 }
 
+// One CTA, one thread, one barrier that nobody ever arrives at: the bounded wait of the GEMM pipeline runs out after
+// `limit_ns` and the kernel reports it the way the pipeline does (STATUS_TIMEOUT in the status word).  Nothing else is
+// in flight: no copy, no TMEM, no second CTA.
+__global__ void wait_selftest_kernel(unsigned long long limit_ns, int32_t* status, unsigned long long* waited_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int s_abort;
+  s_abort = 0;
+  const uint32_t b = ptx::smem_u32(&bar);
+  ptx::mbar_init(b, 1);
+  ptx::fence_mbar_init();
+  const uint64_t t0 = ptx::globaltimer_ns();
+  const bool arrived = ptx::mbar_wait_bounded(b, 0u, &s_abort, limit_ns);
+  *waited_ns = ptx::globaltimer_ns() - t0;
+  if (!arrived) atomicOr(status, STATUS_TIMEOUT);
+}
+
+cudaError_t launch_wait_selftest(grouter_ctx* ctx, unsigned long long limit_ns, unsigned long long* d_waited_ns, cudaStream_t st) {
+  wait_selftest_kernel<<<1, 1, 0, st>>>(limit_ns, ctx->pp.status, d_waited_ns);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,
                               cudaStream_t st) {
   GemmParams p{};
@@ -882,6 +937,7 @@ cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, 
   p.tiles_n = cdiv(N, BN);
   p.status = status;
   p.out_f = C;
+  p.wait_limit_ns = DEFAULT_WAIT_LIMIT_NS;
   Maps m;
   const bool ok = (a_mn ? make_map(&m.A, A, K, M, 64) : make_map(&m.A, A, M, K, 128)) &&
                   (b_mn ? make_map(&m.B, B, K, N, 64) : make_map(&m.B, B, N, K, 128));

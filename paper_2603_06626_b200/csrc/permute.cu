@@ -164,6 +164,30 @@ __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bf
   }
 }
 
+// out = bf16(in), eight elements per thread and pass (the last step of the fused combine).
+__global__ void __launch_bounds__(MOVE_THREADS) cast_rows_kernel(const float4* __restrict__ in, uint4* __restrict__ out, size_t n8) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (size_t)gridDim.x * blockDim.x) {
+    const float4 a = in[2 * i], b = in[2 * i + 1];
+    uint4 v;
+    __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&v);
+    p[0] = __floats2bfloat162_rn(a.x, a.y);
+    p[1] = __floats2bfloat162_rn(a.z, a.w);
+    p[2] = __floats2bfloat162_rn(b.x, b.y);
+    p[3] = __floats2bfloat162_rn(b.z, b.w);
+    out[i] = v;
+  }
+}
+
+cudaError_t launch_cast_rows(grouter_ctx* ctx, const float* in, __nv_bfloat16* out, size_t n, cudaStream_t st) {
+  const size_t n8 = n / 8;
+  size_t want = (n8 + MOVE_THREADS - 1) / MOVE_THREADS;
+  const size_t cap = (size_t)ctx->num_sms * 8;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  cast_rows_kernel<<<(unsigned)want, MOVE_THREADS, 0, st>>>(reinterpret_cast<const float4*>(in), reinterpret_cast<uint4*>(out), n8);
+  return cudaGetLastError();
+}
+
 __global__ void idle_kernel(unsigned long long nanoseconds) {
   unsigned long long t0, t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));

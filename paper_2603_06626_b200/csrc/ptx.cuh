@@ -218,6 +218,11 @@ __device__ __forceinline__ void st_global_v2_stream(float* p, uint32_t a, uint32
 __device__ __forceinline__ void red_add_v2_f32(float* p, uint32_t a, uint32_t b) {
   asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)) : "memory");
 }
+__device__ __forceinline__ void red_add_v4_f32(float* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
+               "f"(__uint_as_float(c)), "f"(__uint_as_float(d))
+               : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory operand descriptor for tcgen05.mma, 128-byte swizzle.

@@ -29,12 +29,12 @@ def rows_ok(name, got, want):
     return worst
 
 
-def run_gpu(w, li, gate_f32=False, idx_i32=False):
+def run_gpu(w, li, gate_f32=False, idx_i32=False, flags=0):
     """One plan + fwd + bwd through the C ABI.  Returns device tensors."""
     from paper_2603_06626_b200 import binding
     layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k, E_tgt=w.E_tgt,
                                  idx_dtype=binding.IDX_I32 if idx_i32 else binding.IDX_U8,
-                                 gate_dtype=binding.GATE_F32 if gate_f32 else binding.GATE_BF16)
+                                 gate_dtype=binding.GATE_F32 if gate_f32 else binding.GATE_BF16, flags=flags)
     idx = to_dev(li.idx.astype(np.int32) if idx_i32 else li.idx)
     fm = None if li.fold_map is None else to_dev(li.fold_map)
     gates = bits_to_bf16(li.gates)
@@ -192,6 +192,31 @@ def test_f32_gates_i32_idx_and_fold_collisions():
     li = synth.make_layer_inputs(w)
     out = run_gpu(w, li, gate_f32=True, idx_i32=True)
     print(check_full(w, li, out))
+
+
+@pytest.mark.parametrize("case", ["tiny", "small", "ragged", "fold", "paper_shape"])
+def test_fused_combine_variant_full_parity(case):
+    """GROUTER_FLAG_FUSED_COMBINE: the down product adds its gate-weighted rows straight into the tokens' fp32 rows.
+    Same bar against the oracle as the two-kernel form; the backward pass is untouched and checked along."""
+    from paper_2603_06626_b200 import binding
+    kw = {}
+    if case in ("tiny", "small"):
+        w = synth.WORKLOADS[case]
+    elif case == "ragged":
+        w = synth.custom_workload("edge", T=257, d=128, ffn=72, E=5, k=3, seed=385)
+    elif case == "paper_shape":
+        w = synth.custom_workload("edge", T=640, d=384, ffn=344, E=128, k=8, seed=1024)
+    else:
+        w = synth.custom_workload("fold", T=700, d=256, ffn=256, E=24, k=4, E_tgt=5, fold_mod=5, seed=11)
+        kw = dict(gate_f32=True, idx_i32=True)
+    li = synth.make_layer_inputs(w)
+    fused = run_gpu(w, li, flags=binding.FLAG_FUSED_COMBINE, **kw)
+    print(check_full(w, li, fused))
+    plain = run_gpu(w, li, **kw)
+    # the two forms round differently (one bf16 rounding of the fp32 sum against k roundings of the rows): close, not equal
+    assert orc.rel_frobenius(f64(fused["Y"]), f64(plain["Y"])) < 8e-3
+    for name in ("dX", "dgates"):
+        assert torch.equal(fused[name], plain[name]), name
 
 
 def test_dense_special_case_unit_gate():
