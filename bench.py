@@ -226,6 +226,84 @@ def combine_ab_leg(dev, w, layer, idx, fm, gates, X, W_gu, W_d, rounds=5, per_ro
             "fused_over_separate": med["fused"] / med["separate"], "rounds": rounds, "forwards_per_round": per_round}
 
 
+def run_expert_parallel(args, rank, local_rank, world, dev):
+    """--parallelism ep: every rank keeps its own T tokens and 1/N of the experts; routed rows travel to the experts'
+    rank and back (NCCL all-to-all into the receiver's own memory, split sizes from the plans' counts, which are gathered
+    once ahead of the timed steps: the routing is known before the step).  With one rank the exchanges are local copies."""
+    import torch
+    import torch.distributed as dist
+    from paper_2603_06626_b200 import binding, ep
+    base = synth.WORKLOADS[args.workload]
+    w = shard.rank_workload(base, rank)
+    if base.E_tgt % world:
+        raise SystemExit(f"--parallelism ep needs E_tgt ({base.E_tgt}) divisible by the number of ranks ({world})")
+    li = synth.make_layer_inputs(w, with_weights=False)
+    owner = np.arange(base.E_tgt) // (base.E_tgt // world)
+    relabel, first = ep.relabel_experts(owner, world)
+    fm = relabel if li.fold_map is None else relabel[li.fold_map]
+    fold = torch.from_numpy(np.ascontiguousarray(fm, dtype=np.int32)).to(dev)
+
+    def bf16(a):
+        return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(dev).view(torch.bfloat16)
+
+    mine = range(int(first[rank]), int(first[rank + 1]))          # identity relabelling: new id == old id
+    W_gu = bf16(np.stack([synth.expert_W_gu(base, e) for e in mine]))
+    W_d = bf16(np.stack([synth.expert_W_d(base, e) for e in mine]))
+    idx, gates, X, dY = torch.from_numpy(li.idx).to(dev), bf16(li.gates), bf16(li.X), bf16(li.dY)
+    r = ep.ExpertParallelRank(rank, world, w.T, w.d, w.ffn, w.E_src, w.E_tgt, w.k, first, device=str(dev))
+    counts = r.plan(idx, fold)
+    if world > 1:
+        allc = [torch.empty_like(counts) for _ in range(world)]
+        dist.all_gather(allc, counts)
+        counts_all = torch.stack(allc).cpu().numpy()
+    else:
+        counts_all = counts.cpu().numpy()[None, :]
+    r.set_counts(counts_all)
+    Y, dX = torch.empty_like(X), torch.empty_like(X)
+    dg = torch.empty((w.T, w.k), dtype=torch.float32, device=dev)
+    dW_gu = torch.empty(W_gu.shape, dtype=torch.float32, device=dev)
+    dW_d = torch.empty(W_d.shape, dtype=torch.float32, device=dev)
+
+    def step():
+        r.plan(idx, fold)
+        r.run_step(X, dY, gates, W_gu, W_d, Y, dX, dg, dW_gu, dW_d)
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step()
+    shard.barrier(world)
+    torch.cuda.synchronize()
+    wall0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    wall1 = time.time()
+    shard.barrier(world)
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+    ms_step = shard.max_over_ranks(e0.elapsed_time(e1), dev, world) / args.steps
+    assert r.src.status() == 0 and (r.exp is None or r.exp.status() == 0)
+    rows_out = int(r.layout["send_counts"].sum() - r.layout["send_counts"][rank])
+    if rank == 0:
+        peaks, peak_src = load_peaks()
+        flops_rank = 18.0 * w.d * w.ffn * float(r.n_recv)
+        line = {"metric": METRIC, "value": shard.job_tokens_per_sec(world, w.T, ms_step), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "bf16", "data": "synthetic", "config": dict(workload_config(base, world), parallelism=f"ep{world}"),
+                "clocks": clocks, "gpu_launches": int((3 + 4 + 5 + 3 + 7) * args.steps),
+                "roofline": {"bound": "tensor", "achieved": flops_rank / (ms_step * 1e-3) / 1e12, "peak": peaks["bf16_tflops_sustained"],
+                             "unit": "TFLOP/s", "frac": flops_rank / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], "traffic": None,
+                             "peak_source": f"{peak_src} cuBLAS bf16, sustained; the whole step (exchanges included) of rank 0's experts"},
+                "exchange": {"rows_sent_to_other_ranks_per_direction": rows_out, "bytes_per_step": 4.0 * rows_out * w.d * 2,
+                             "transfers_per_step": 4, "split_sizes": "from the plans' counts, gathered once before the timed steps"}}
+        print(json.dumps(line))
+    r.close()
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -389,6 +467,7 @@ def run_reference(args):
 def workload_config(w: synth.Workload, n_gpus: int):
     return {"workload": w.name, "T": w.T, "d": w.d, "ffn": w.ffn, "E_src": w.E_src, "E_tgt": w.E_tgt, "k": w.k, "load": w.load,
             "zipf_s": w.zipf_s, "tokens_per_gpu": w.T, "global_tokens": w.T * n_gpus, "parallelism": f"dp{n_gpus}",
+            "dw_allreduce_in_step": False,
             "l2": "working set (weights + expert-ordered activations, several GB) exceeds the 126 MB L2"
             if w.name in ("skewed", "large", "fine_fold", "small") else "fits L2: flushed between steps"}
 
@@ -400,6 +479,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="large", choices=list(synth.WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--parallelism", default="dp", choices=["dp", "ep"],
+                    help="dp: token-sharded replicas (default); ep: experts split over the ranks, routed rows exchanged")
+    ap.add_argument("--dw-allreduce", action="store_true",
+                    help="dp with more than one rank: all-reduce the weight gradients inside every timed step")
     ap.add_argument("--cpu-baseline-experts", type=int, default=12, help="whole experts the CPU baseline times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -424,6 +507,11 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     warm = max(args.warmup, 3)
+    if args.parallelism == "ep":
+        run_expert_parallel(args, rank, local_rank, world, dev)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     base = synth.WORKLOADS[args.workload]
     w = shard.rank_workload(base, rank)
@@ -449,6 +537,9 @@ def main():
         layer.plan(idx, fm)
         layer.forward(X, gates, W_gu, W_d, Y)
         layer.backward(dY, X, gates, W_gu, W_d, dX, dW_gu, dW_d, dgates)
+        if args.dw_allreduce and world > 1:       # the one collective data parallelism adds: summed weight gradients
+            dist.all_reduce(dW_gu)
+            dist.all_reduce(dW_d)
 
     def barrier():
         shard.barrier(world)
@@ -634,7 +725,7 @@ def main():
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
         "ms_per_step": ms_step, "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_best": step_ms[0], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic", "config": workload_config(base, world), "clocks": clocks,
+        "data": "synthetic", "config": dict(workload_config(base, world), dw_allreduce_in_step=bool(args.dw_allreduce and world > 1)), "clocks": clocks,
         "gpu_launches": int(sum(v[1] for v in per_kernel.values()) // max(n_timed, 1) * args.steps), "roofline": roofline, "kernels": kernels, "gemm_summary": summary, "plan": plan,
         "gemm_cycles": gemm_cycles,
         "load_stats": synth.load_stats(li.idx, li.fold_map, w.E_tgt),

@@ -189,6 +189,45 @@ int grouter_routing_stats(const void* idx, int32_t idx_dtype, int32_t T, int32_t
  * group j.  Needs E_tgt <= E_src.  Plain host arrays; no GPU work. */
 int grouter_fold_greedy_host(const int32_t* coact_host, int32_t E_src, int32_t E_tgt, int32_t* fold_map_host);
 
+/* ---- Expert parallelism (section "Decoupling Communication Optimization"; appendix "Efficiency Experiment Detail") ----
+ * Experts are split over `world` ranks; every rank keeps its own tokens, and routed rows travel to the rank that owns
+ * their expert and back.  With preemptive routing all per-peer row counts follow from the per-rank expert histograms
+ * (grouter_plan's `counts` of every rank, known before the step from the routing cache), so the transfer needs no
+ * size exchange.  These calls do everything around the transfer; the transfer is the caller's collective (e.g. an
+ * NCCL all-to-all with the split sizes below) into the receiver's own memory.
+ *
+ * grouter_ep_relabel_host (host): renumbers the experts so that every rank owns a contiguous range.
+ *   expert_rank [E] in [0,world): owner of each expert (any assignment, e.g. the paper's expert grouping)
+ *   relabel [E] out: new id of each expert (ranks ascending, old order kept within a rank); compose it with the fold
+ *           map (fold_map'[i] = relabel[fold_map[i]]) and store the weights in the new order
+ *   first_expert [world+1] out: rank r owns new ids first_expert[r] .. first_expert[r+1]-1
+ * grouter_ep_layout_host (host): per-peer counts and offsets for rank `rank`, in rows.
+ *   counts_all [world,E]: row q = `counts` of rank q's plan (new ids)
+ *   send_counts/send_offsets [world]/[world+1]: the rows for peer p are rows send_offsets[p] .. of this rank's
+ *           expert-ordered rows (grouter_ep_dispatch_rows writes them in exactly that order)
+ *   recv_counts/recv_offsets [world]/[world+1]: rows arriving from peer q land at recv_offsets[q]
+ *   recv_seg_offsets [world*n_local+1], n_local = experts of `rank`: exclusive prefix of the (source rank, local expert)
+ *           segments of the received rows
+ * grouter_ep_expand_ids (device): idx_out[r] = local expert (0..n_local-1) of received row r, from recv_seg_offsets on
+ *   the device; the receiving rank then runs grouter_plan / fwd / bwd on the received rows as T = rows, k = 1, unit gates.
+ * grouter_ep_dispatch_rows (device): rows[slot_to_row[s], :] = gate_s * src[token of s, :]  (gates NULL: plain copy).
+ *   rows [T*k, d] bf16, expert-ordered and unpadded.  Forward: src = X, no gates.  Backward: src = dY with the gates.
+ * grouter_ep_combine_rows (device): out[t,:] = sum_j gate * rows[slot_to_row[t*k+j], :] in fp32, slot order (gates NULL:
+ *   plain sum), and/or dgates[t,j] = <dY[t,:], rows[slot_to_row[t*k+j], :]>.  out or dgates may be NULL (not both).
+ *   Forward: rows = returned expert outputs, with the gates -> Y (Eq. 1).  Backward: rows = returned input gradients,
+ *   no gates -> dX; dgates from the forward's returned rows and dY.
+ * The two row calls need a prior grouter_plan on ctx (they read its slot_to_row) and use ctx's T, k, d, gate_dtype.
+ * Errors: INVALID_ARG, MISALIGNED, INVALID_STATE, UNSUPPORTED, CUDA. */
+int grouter_ep_relabel_host(int32_t E, int32_t world, const int32_t* expert_rank, int32_t* relabel, int32_t* first_expert);
+int grouter_ep_layout_host(int32_t world, int32_t rank, int32_t E, const int32_t* first_expert, const int32_t* counts_all,
+                           int32_t* send_counts, int32_t* send_offsets, int32_t* recv_counts, int32_t* recv_offsets,
+                           int32_t* recv_seg_offsets);
+int grouter_ep_expand_ids(const int32_t* seg_offsets, int32_t n_seg, int32_t n_local, int32_t n_rows, int32_t idx_dtype, void* idx_out,
+                          void* stream);
+int grouter_ep_dispatch_rows(grouter_ctx* ctx, const void* src, const void* gates, void* rows, void* stream);
+int grouter_ep_combine_rows(grouter_ctx* ctx, const void* rows, const void* gates, void* out, const void* dY, float* dgates,
+                            void* stream);
+
 /* Forward, Eq. 1:  Y[t,:] = sum_j gates[t,j] * f_{e(t,j)}(X[t,:]).
  *   X     [T,d] bf16             gates [T,k] bf16 or f32 (dims.gate_dtype), used as given
  *   W_gu  [E_tgt, 2*ffn, d] bf16: rows 0..ffn-1 gate projection, ffn..2ffn-1 up projection

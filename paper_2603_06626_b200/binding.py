@@ -23,7 +23,8 @@ GATE_BF16, GATE_F32 = 0, 1
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
-           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest"]
+           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest",
+           "grouter_ep_relabel_host", "grouter_ep_layout_host", "grouter_ep_expand_ids", "grouter_ep_dispatch_rows", "grouter_ep_combine_rows"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW", "plan_scan"]
 
@@ -95,6 +96,16 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_gemm_cycles_read.restype = ctypes.c_int
     lib.grouter_wgrad_chunk_rows.argtypes = [vp]
     lib.grouter_wgrad_chunk_rows.restype = ctypes.c_int32
+    lib.grouter_ep_relabel_host.argtypes = [ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+    lib.grouter_ep_relabel_host.restype = ctypes.c_int
+    lib.grouter_ep_layout_host.argtypes = [ctypes.c_int32] * 3 + [vp] * 7
+    lib.grouter_ep_layout_host.restype = ctypes.c_int
+    lib.grouter_ep_expand_ids.argtypes = [vp] + [ctypes.c_int32] * 4 + [vp, vp]
+    lib.grouter_ep_expand_ids.restype = ctypes.c_int
+    lib.grouter_ep_dispatch_rows.argtypes = [vp] * 5
+    lib.grouter_ep_dispatch_rows.restype = ctypes.c_int
+    lib.grouter_ep_combine_rows.argtypes = [vp] * 7
+    lib.grouter_ep_combine_rows.restype = ctypes.c_int
     lib.grouter_set_wait_limit.argtypes = [vp, ctypes.c_int64]
     lib.grouter_set_wait_limit.restype = ctypes.c_int
     lib.grouter_wait_selftest.argtypes = [vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64), vp]
@@ -224,6 +235,16 @@ class GrouterLayer:
         names = ["gemm_up_swiglu", "gemm_down", "gemm_dH", "gemm_dX", "wgrad_down", "wgrad_gate_up"]
         keys = ["cycles", "wait_operands", "wait_accumulator", "tiles", "k_steps"]
         return {n: {k: int(buf[5 * i + j]) for j, k in enumerate(keys)} for i, n in enumerate(names)}
+
+    def ep_dispatch_rows(self, src, gates, rows):
+        """rows[slot_to_row[s], :] = gate_s * src[token of s, :] (gates None: copy); rows [T*k, d] bf16."""
+        _check(self.lib.grouter_ep_dispatch_rows(self.ctx, _ptr(src), _ptr(gates), _ptr(rows), _stream()), "grouter_ep_dispatch_rows")
+        return rows
+
+    def ep_combine_rows(self, rows, gates=None, out=None, dY=None, dgates=None):
+        """out[t, :] = sum_j gate * rows[slot_to_row[t*k+j], :] and/or dgates[t, j] = <dY[t, :], rows[slot_to_row[t*k+j], :]>."""
+        _check(self.lib.grouter_ep_combine_rows(self.ctx, _ptr(rows), _ptr(gates), _ptr(out), _ptr(dY), _ptr(dgates), _stream()),
+               "grouter_ep_combine_rows")
 
     def set_wait_limit(self, microseconds: int) -> None:
         """Limit of every bounded device-side wait of this context's later launches."""

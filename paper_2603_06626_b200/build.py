@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgrouter.so")
-SOURCES = ["api.cu", "plan.cu", "permute.cu", "gemm.cu", "route.cu", "stats.cu"]
+SOURCES = ["api.cu", "plan.cu", "permute.cu", "gemm.cu", "route.cu", "stats.cu", "ep.cu"]
 
 
 def _newest_source_mtime() -> float:

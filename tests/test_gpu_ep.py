@@ -1,0 +1,121 @@
+"""The expert-parallel data path on one GPU against the oracle.
+
+Four ranks are emulated in one process, one after the other (none of their kernels waits on another rank): every
+rank object runs its phases, and the all-to-all between phases is emulated by copying each (source, destination)
+block between the ranks' buffers with the split sizes the library computed.  The result must be the layer of Eq. 1
+over every rank's tokens, and every expert's weight gradient must be the sum over the tokens of all ranks."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import grouter_oracle as orc
+from paper_2603_06626_b200 import synth
+from tests.gpu_util import bits_to_bf16, to_dev
+
+pytestmark = pytest.mark.gpu
+TOL, ROW_TOL = 1e-2, 3e-2
+
+
+def _exchange(ranks, src_name, dst_name, to_experts):
+    """dst buffer of rank p, block of source q  <-  src buffer of rank q, block for p (or the reverse direction)."""
+    for p, rp in enumerate(ranks):
+        for q, rq in enumerate(ranks):
+            if to_experts:
+                n = int(rq.layout["send_counts"][p])
+                assert n == int(rp.layout["recv_counts"][q])
+                so, ro = int(rq.layout["send_offsets"][p]), int(rp.layout["recv_offsets"][q])
+                getattr(rp, dst_name)[ro:ro + n].copy_(getattr(rq, src_name)[so:so + n])
+            else:
+                n = int(rq.layout["recv_counts"][p])
+                so, ro = int(rq.layout["recv_offsets"][p]), int(rp.layout["send_offsets"][q])
+                getattr(rp, dst_name)[ro:ro + n].copy_(getattr(rq, src_name)[so:so + n])
+
+
+def test_expert_parallel_step_four_emulated_ranks_matches_oracle():
+    from paper_2603_06626_b200 import ep
+    world, d, F, E, k = 4, 128, 192, 12, 3
+    Ts = [320, 257, 400, 96]
+    owner = np.array([(5 * e + 1) % world for e in range(E)])
+    owner[owner == 3] = 2                                   # rank 3 owns no expert: it only sends and receives its own rows back
+    relabel, first = ep.relabel_experts(owner, world)
+    base = synth.custom_workload("ep", T=Ts[0], d=d, ffn=F, E=E, k=k, seed=77)
+    W_gu_bits = np.stack([synth.expert_W_gu(base, e) for e in range(E)])
+    W_d_bits = np.stack([synth.expert_W_d(base, e) for e in range(E)])
+    inv = np.argsort(relabel)                               # new id -> old id
+    W_gu_new, W_d_new = bits_to_bf16(W_gu_bits[inv]), bits_to_bf16(W_d_bits[inv])
+    fold = to_dev(relabel.astype(np.int32))
+    lis, ranks = [], []
+    for q in range(world):
+        w = synth.custom_workload("ep", T=Ts[q], d=d, ffn=F, E=E, k=k, load="zipf", zipf_s=0.9, seed=500 + q)
+        lis.append(synth.make_layer_inputs(w, with_weights=False))
+        ranks.append(ep.ExpertParallelRank(q, world, Ts[q], d, F, E, E, k, first))
+    counts_all = np.stack([r.plan(to_dev(li.idx), fold).cpu().numpy() for r, li in zip(ranks, lis)])
+    for r in ranks:
+        r.set_counts(counts_all)
+        assert r.src.status() == 0
+    assert ranks[3].exp is None and sum(r.n_recv for r in ranks) == sum(Ts) * k
+    dev_in = [dict(X=bits_to_bf16(li.X), dY=bits_to_bf16(li.dY), gates=bits_to_bf16(li.gates)) for li in lis]
+    local_w = [(W_gu_new[first[p]:first[p + 1]], W_d_new[first[p]:first[p + 1]]) for p in range(world)]
+
+    for r, t in zip(ranks, dev_in):
+        r.fwd_dispatch(t["X"])
+    _exchange(ranks, "send_rows", "recv_rows", True)
+    for r, (wg, wd) in zip(ranks, local_w):
+        r.fwd_expert(wg, wd)
+    _exchange(ranks, "out_rows", "fwd_back", False)
+    Ys = [r.fwd_combine(t["gates"]) for r, t in zip(ranks, dev_in)]
+    for r, t in zip(ranks, dev_in):
+        r.bwd_dispatch(t["dY"], t["gates"])
+    _exchange(ranks, "send_rows", "recv_rows2", True)
+    dWs = [r.bwd_expert(wg, wd)[1:] for r, (wg, wd) in zip(ranks, local_w)]
+    _exchange(ranks, "out_rows", "back_rows", False)
+    outs = [r.bwd_combine(t["dY"]) for r, t in zip(ranks, dev_in)]
+    torch.cuda.synchronize()
+    for r in ranks:
+        assert r.src.status() == 0 and (r.exp is None or r.exp.status() == 0)
+
+    f64 = synth.bf16_bits_to_f64
+    weights = orc.Weights(f64(W_gu_bits), f64(W_d_bits))     # the oracle works in the original expert numbering
+    for q, li in enumerate(lis):
+        Y = orc.moe_forward(f64(li.X), li.idx, f64(li.gates), weights, E)
+        dX, dg = orc.moe_backward_tokens(f64(li.dY), f64(li.X), li.idx, f64(li.gates), weights, E)
+        got = dict(Y=Ys[q], dX=outs[q][0], dgates=outs[q][1])
+        for name, want in (("Y", Y), ("dX", dX), ("dgates", dg)):
+            g = got[name].double().cpu().numpy()
+            assert orc.rel_frobenius(g, want) < TOL, (q, name)
+            assert orc.rel_rows(g, want).max() < ROW_TOL, (q, name)
+    X_all = np.concatenate([f64(li.X) for li in lis]); dY_all = np.concatenate([f64(li.dY) for li in lis])
+    idx_all = np.concatenate([li.idx for li in lis]); g_all = np.concatenate([f64(li.gates) for li in lis])
+    for e in range(E):
+        p = int(owner[e])
+        want_gu, want_d = orc.moe_backward_expert(dY_all, X_all, idx_all, g_all, weights, E, e)
+        got_gu = dWs[p][0][relabel[e] - first[p]].double().cpu().numpy()
+        got_d = dWs[p][1][relabel[e] - first[p]].double().cpu().numpy()
+        assert orc.rel_frobenius(got_gu, want_gu) < TOL and orc.rel_frobenius(got_d, want_d) < TOL, e
+    for r in ranks:
+        r.close()
+
+
+def test_expert_parallel_run_step_world_one_equals_the_plain_layer():
+    """world = 1: the exchanges are local copies; the step through the expert-parallel wiring agrees with the oracle."""
+    from paper_2603_06626_b200 import ep
+    w = synth.custom_workload("ep1", T=300, d=256, ffn=128, E=6, k=2, seed=9)
+    li = synth.make_layer_inputs(w)
+    relabel, first = ep.relabel_experts(np.zeros(w.E_tgt, dtype=np.int32), 1)
+    r = ep.ExpertParallelRank(0, 1, w.T, w.d, w.ffn, w.E_src, w.E_tgt, w.k, first)
+    counts = r.plan(to_dev(li.idx), None).cpu().numpy()
+    r.set_counts(counts[None, :])
+    X, dY, gates = bits_to_bf16(li.X), bits_to_bf16(li.dY), bits_to_bf16(li.gates)
+    Y, dX, dg, dW_gu, dW_d = r.run_step(X, dY, gates, bits_to_bf16(li.W_gu), bits_to_bf16(li.W_d))
+    torch.cuda.synchronize()
+    f64 = synth.bf16_bits_to_f64
+    weights = orc.Weights(f64(li.W_gu), f64(li.W_d))
+    Yo = orc.moe_forward(f64(li.X), li.idx, f64(li.gates), weights, w.E_tgt)
+    dXo, dgo, dWo = orc.moe_backward(f64(li.dY), f64(li.X), li.idx, f64(li.gates), weights, w.E_tgt)
+    assert orc.rel_frobenius(Y.double().cpu().numpy(), Yo) < TOL
+    assert orc.rel_frobenius(dX.double().cpu().numpy(), dXo) < TOL
+    assert orc.rel_frobenius(dg.double().cpu().numpy(), dgo) < TOL
+    for e in range(w.E_tgt):
+        assert orc.rel_frobenius(dW_gu[e].double().cpu().numpy(), dWo[e][0]) < TOL
+        assert orc.rel_frobenius(dW_d[e].double().cpu().numpy(), dWo[e][1]) < TOL
+    r.close()
