@@ -158,7 +158,8 @@ def router_head_leg(dev, T=32768, d_h=512, E_src=128, E_tgt=128, k=8, iters=20):
     ms = e0.elapsed_time(e1) / iters
     by = T * d_h * 2.0 + E_src * d_h * 2.0 + 3.0 * k * T
     return {"T": T, "d_h": d_h, "E": E_src, "k": k, "ms": ms, "tokens_per_s": T / (ms * 1e-3), "algorithmic_bytes": by,
-            "gbs": by / (ms * 1e-3) / 1e9, "gpu_launches_per_call": 2}
+            "gbs": by / (ms * 1e-3) / 1e9,
+            "gpu_launches_per_call": 1 if (E_src <= 256 and k <= 8) else 2}
 
 
 def routing_stats_leg(dev, idx, E, seq_len=4096, n_nodes=8, iters=20):

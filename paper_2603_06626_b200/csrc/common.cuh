@@ -160,6 +160,8 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
 cudaError_t launch_zero_split_dw(grouter_ctx* ctx, float* dW_gu, float* dW_d, cudaStream_t st);
 // A kernel that only lets `microseconds` pass (one thread watching the global timer, capped at one second).
 cudaError_t launch_idle(int microseconds, cudaStream_t st);
+// Tensor map of a row-major bf16 matrix [rows, cols] for 128-byte-swizzled tiles of 64 columns x box_rows rows.
+bool make_bf16_tile_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 // Measures one bounded wait that cannot succeed (see grouter_wait_selftest).
 cudaError_t launch_wait_selftest(grouter_ctx* ctx, unsigned long long limit_ns, unsigned long long* d_waited_ns, cudaStream_t st);
 cudaError_t launch_dense_gemm(const void* A, int a_mn, const void* B, int b_mn, float* C, int M, int N, int K, int32_t* status,

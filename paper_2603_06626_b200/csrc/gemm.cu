@@ -765,6 +765,10 @@ static bool make_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t 
   return r == CUDA_SUCCESS;
 }
 
+bool make_bf16_tile_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  return make_map(tm, base, rows, cols, box_rows);
+}
+
 struct Maps {
   CUtensorMap A, B, C0, C1, C2;
 };
