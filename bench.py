@@ -576,13 +576,33 @@ def main():
     value = shard.job_tokens_per_sec(world, w.T, ms_step)
 
     # ---- the per-kernel table: a pass of its own with an event pair around every launch (not part of `value`) ----
+    # (with every kernel in line on the one stream: the event pairs then bracket one kernel each)
     n_table = min(args.steps, 10)
+    layer.set_overlap(False)
     layer.timing_enable(len(binding.KERNEL_SLOTS) * n_table)
     for _ in range(n_table):
         step()
     per_kernel = layer.timing_read()
     layer.timing_enable(0)
     layer.check_status()
+    # what running the backward pass's two bandwidth-bound kernels beside the GEMMs is worth: whole steps, interleaved
+    overlap_ab = None
+    if world == 1 and not args.no_isolated:
+        t_ab = {True: [], False: []}
+        for _ in range(3):
+            for on in (True, False):
+                layer.set_overlap(on)
+                step()
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a0.record()
+                for _ in range(5):
+                    step()
+                a1.record()
+                torch.cuda.synchronize()
+                t_ab[on].append(a0.elapsed_time(a1) / 5)
+        overlap_ab = {"step_ms_beside_gemms": statistics.median(t_ab[True]), "step_ms_in_line": statistics.median(t_ab[False]),
+                      "rounds": 3, "steps_per_round": 5}
+    layer.set_overlap(True)
     # the plan build alone, back to back on the stream (its three launches are too short for event pairs around each)
     pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     pe0.record()
@@ -595,6 +615,7 @@ def main():
     # ---- every kernel alone: 30 ms of idle time after each launch, so that none starts at the power cap ----
     isolated = None
     if world == 1 and not args.no_isolated:
+        layer.set_overlap(False)
         layer.timing_gap(30000)
         layer.timing_enable(len(binding.KERNEL_SLOTS) * 3)
         for _ in range(3):
@@ -602,6 +623,7 @@ def main():
         isolated = layer.timing_read()
         layer.timing_enable(0)
         layer.timing_gap(0)
+        layer.set_overlap(True)
         layer.check_status()
 
     # ---- where the issuers' cycles go (a few steps with the accounting on; not part of any timed number) ----
@@ -728,7 +750,7 @@ def main():
         "ms_per_step": ms_step, "ms_per_step_median": step_ms[len(step_ms) // 2], "ms_per_step_best": step_ms[0], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": dict(workload_config(base, world), dw_allreduce_in_step=bool(args.dw_allreduce and world > 1)), "clocks": clocks,
         "gpu_launches": int(sum(v[1] for v in per_kernel.values()) // max(n_timed, 1) * args.steps), "roofline": roofline, "kernels": kernels, "gemm_summary": summary, "plan": plan,
-        "gemm_cycles": gemm_cycles,
+        "gemm_cycles": gemm_cycles, "overlap_ab": overlap_ab,
         "load_stats": synth.load_stats(li.idx, li.fold_map, w.E_tgt),
     }
     if e2e is not None:

@@ -251,6 +251,12 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
                     const void* W_d, void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace,
                     void* stream);
 
+/* grouter_moe_bwd runs two bandwidth-bound kernels (the zero-fill of split experts' gradients, the final reduction of
+ * dX) on a stream the context owns, beside the tensor-core products they do not depend on, and joins them back into
+ * `stream` before it returns: to the caller the call is ordered on `stream` as ever.  on = 0 puts them back in line
+ * (measurement aid; the default is on).  No counterpart in the paper. */
+int grouter_set_overlap(grouter_ctx* ctx, int32_t on);
+
 /* Longest run of an expert's rows that the weight-gradient products of grouter_moe_bwd contract in one piece (host
  * only; a power of two between 1024 and 16384 fixed at grouter_create from the dims and the device's SM count: as long
  * as possible, shorter when the per-expert gradient matrices are too small to keep every SM busy otherwise).  The

@@ -23,7 +23,7 @@ GATE_BF16, GATE_F32 = 0, 1
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
-           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest",
+           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest", "grouter_set_overlap",
            "grouter_ep_relabel_host", "grouter_ep_layout_host", "grouter_ep_expand_ids", "grouter_ep_dispatch_rows", "grouter_ep_combine_rows"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW", "plan_scan"]
@@ -106,6 +106,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_ep_dispatch_rows.restype = ctypes.c_int
     lib.grouter_ep_combine_rows.argtypes = [vp] * 7
     lib.grouter_ep_combine_rows.restype = ctypes.c_int
+    lib.grouter_set_overlap.argtypes = [vp, ctypes.c_int32]
+    lib.grouter_set_overlap.restype = ctypes.c_int
     lib.grouter_set_wait_limit.argtypes = [vp, ctypes.c_int64]
     lib.grouter_set_wait_limit.restype = ctypes.c_int
     lib.grouter_wait_selftest.argtypes = [vp, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64), vp]
@@ -245,6 +247,10 @@ class GrouterLayer:
         """out[t, :] = sum_j gate * rows[slot_to_row[t*k+j], :] and/or dgates[t, j] = <dY[t, :], rows[slot_to_row[t*k+j], :]>."""
         _check(self.lib.grouter_ep_combine_rows(self.ctx, _ptr(rows), _ptr(gates), _ptr(out), _ptr(dY), _ptr(dgates), _stream()),
                "grouter_ep_combine_rows")
+
+    def set_overlap(self, on: bool) -> None:
+        """Bandwidth-bound kernels of the backward pass beside the GEMMs (default) or in line."""
+        _check(self.lib.grouter_set_overlap(self.ctx, 1 if on else 0), "grouter_set_overlap")
 
     def set_wait_limit(self, microseconds: int) -> None:
         """Limit of every bounded device-side wait of this context's later launches."""

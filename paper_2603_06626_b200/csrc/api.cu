@@ -181,11 +181,23 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->d_cycles = nullptr;
   c->wait_limit_ns = DEFAULT_WAIT_LIMIT_NS;
   c->d_waited = nullptr;
-  c->s_in = c->s_out = nullptr;
+  c->s_in = c->s_out = c->s_side = nullptr;
+  c->ev_fork = c->ev_zero_done = c->ev_dx_done = c->ev_join = c->ev_plan_done = c->ev_dy_gathered = c->ev_down_done = c->ev_combined = nullptr;
+  c->step_combine_on_side = c->step_dy_pregathered = false;
+  c->overlap = true;
   for (int i = 0; i < 2; ++i) c->ev_in_fwd[i] = c->ev_in_bwd[i] = c->ev_fwd_done[i] = c->ev_bwd_done[i] = c->ev_out_done[i] = nullptr;
   {
     bool ok = cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking) == cudaSuccess;
+              cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&c->s_side, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_zero_done, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_dx_done, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_plan_done, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_dy_gathered, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_down_done, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&c->ev_combined, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; i < 2 && ok; ++i)
       ok = cudaEventCreateWithFlags(&c->ev_in_fwd[i], cudaEventDisableTiming) == cudaSuccess &&
            cudaEventCreateWithFlags(&c->ev_in_bwd[i], cudaEventDisableTiming) == cudaSuccess &&
@@ -241,6 +253,9 @@ void grouter_destroy(grouter_ctx* ctx) {
   free_events(ctx);
   if (ctx->s_in) cudaStreamDestroy(ctx->s_in);
   if (ctx->s_out) cudaStreamDestroy(ctx->s_out);
+  if (ctx->s_side) cudaStreamDestroy(ctx->s_side);
+  for (cudaEvent_t e : {ctx->ev_fork, ctx->ev_zero_done, ctx->ev_dx_done, ctx->ev_join, ctx->ev_plan_done, ctx->ev_dy_gathered, ctx->ev_down_done, ctx->ev_combined})
+    if (e) cudaEventDestroy(e);
   for (int i = 0; i < 2; ++i) {
     cudaEvent_t evs[5] = {ctx->ev_in_fwd[i], ctx->ev_in_bwd[i], ctx->ev_fwd_done[i], ctx->ev_bwd_done[i], ctx->ev_out_done[i]};
     for (cudaEvent_t e : evs)
@@ -309,7 +324,17 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
       Timed tm(ctx, 4, st);
       if (launch_grouped_gemm(ctx, MODE_DOWN, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
     }
-    {
+    if (ctx->step_combine_on_side) {
+      // (step call only) the combine runs beside the backward pass's first kernels; whoever needs Y or overwrites the
+      // expert outputs waits for ev_combined
+      if (cudaEventRecord(ctx->ev_down_done, st) != cudaSuccess || cudaStreamWaitEvent(ctx->s_side, ctx->ev_down_done, 0) != cudaSuccess)
+        return GROUTER_ERR_CUDA;
+      {
+        Timed tm(ctx, 5, ctx->s_side);
+        if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, ctx->s_side) != cudaSuccess) return GROUTER_ERR_CUDA;
+      }
+      if (cudaEventRecord(ctx->ev_combined, ctx->s_side) != cudaSuccess) return GROUTER_ERR_CUDA;
+    } else {
       Timed tm(ctx, 5, st);
       if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(Y), nullptr, 0, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
     }
@@ -328,7 +353,26 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Workspace ws = carve_workspace(ctx->dims, ctx->R_pad_max, workspace);
   const int n_part = 2 * ((ctx->dims.ffn + 255) / 256);  // two column halves per 256-wide tile
+  // Two bandwidth-bound kernels have no business on the GEMMs' critical path: the zero-fill of split experts' gradients
+  // (needs only the plan) and the final reduction of dX (needs the dX product, not the last weight gradient).  They run
+  // on a stream of the context beside the GEMMs, forked from and joined back into the caller's stream with events, so
+  // the caller sees one ordered call (the pattern is capturable in a CUDA graph).
+  const bool side = ctx->overlap && ctx->idle_gap_us == 0;
+  cudaStream_t ss = side ? ctx->s_side : st;
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+  if (side) {
+    if (!ok(cudaEventRecord(ctx->ev_fork, st)) || !ok(cudaStreamWaitEvent(ss, ctx->ev_fork, 0))) return GROUTER_ERR_CUDA;
+  }
   {
+    Timed tm(ctx, 12, ss);
+    // (when accumulating, the caller's gradients are the starting value of every expert's sum: nothing to zero)
+    if (!(ctx->dims.flags & GROUTER_FLAG_ACCUMULATE_DW) && launch_zero_split_dw(ctx, dW_gu, dW_d, ss) != cudaSuccess)
+      return GROUTER_ERR_CUDA;
+  }
+  if (side && !ok(cudaEventRecord(ctx->ev_zero_done, ss))) return GROUTER_ERR_CUDA;
+  if (ctx->step_dy_pregathered) {
+    if (!ok(cudaStreamWaitEvent(st, ctx->ev_dy_gathered, 0))) return GROUTER_ERR_CUDA;
+  } else {
     Timed tm(ctx, 6, st);
     if (launch_scatter_rows(ctx, static_cast<const __nv_bfloat16*>(dY), ws.dYp, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
@@ -336,29 +380,30 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
     Timed tm(ctx, 7, st);
     if (launch_grouped_gemm(ctx, MODE_DH, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
-  {
-    Timed tm(ctx, 12, st);
-    // (when accumulating, the caller's gradients are the starting value of every expert's sum: nothing to zero)
-    if (!(ctx->dims.flags & GROUTER_FLAG_ACCUMULATE_DW) && launch_zero_split_dw(ctx, dW_gu, dW_d, st) != cudaSuccess)
-      return GROUTER_ERR_CUDA;
-  }
+  if (side && !ok(cudaStreamWaitEvent(st, ctx->ev_zero_done, 0))) return GROUTER_ERR_CUDA;
   {
     Timed tm(ctx, 8, st);
     if (launch_grouped_gemm(ctx, MODE_WGRAD_D, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
+  if (ctx->step_combine_on_side && !ok(cudaStreamWaitEvent(st, ctx->ev_combined, 0))) return GROUTER_ERR_CUDA;   // dXp reuses the expert outputs' buffer
   {
     Timed tm(ctx, 9, st);
     if (launch_grouped_gemm(ctx, MODE_DX, ws, gates, W_gu, W_d, nullptr, nullptr, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
+  if (side) {
+    if (!ok(cudaEventRecord(ctx->ev_dx_done, st)) || !ok(cudaStreamWaitEvent(ss, ctx->ev_dx_done, 0))) return GROUTER_ERR_CUDA;
+  }
+  {
+    Timed tm(ctx, 11, ss);
+    if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(dX), ws.dgate_part, n_part, dgates, ss) != cudaSuccess)
+      return GROUTER_ERR_CUDA;
+  }
+  if (side && !ok(cudaEventRecord(ctx->ev_join, ss))) return GROUTER_ERR_CUDA;
   {
     Timed tm(ctx, 10, st);
     if (launch_grouped_gemm(ctx, MODE_WGRAD_GU, ws, gates, W_gu, W_d, dW_gu, dW_d, st) != cudaSuccess) return GROUTER_ERR_CUDA;
   }
-  {
-    Timed tm(ctx, 11, st);
-    if (launch_reduce_rows(ctx, ws.O, static_cast<__nv_bfloat16*>(dX), ws.dgate_part, n_part, dgates, st) != cudaSuccess)
-      return GROUTER_ERR_CUDA;
-  }
+  if (side && !ok(cudaStreamWaitEvent(st, ctx->ev_join, 0))) return GROUTER_ERR_CUDA;
   return GROUTER_OK;
 }
 
@@ -387,17 +432,35 @@ int grouter_moe_step_host(grouter_ctx* ctx, const void* idx_host, const void* ga
   if (!ok(cudaMemcpyAsync(sb + sg.dY, dY_host, Td * 2, cudaMemcpyHostToDevice, ctx->s_in))) return GROUTER_ERR_CUDA;   // during plan + fwd
   if (!ok(cudaEventRecord(ctx->ev_in_bwd[set], ctx->s_in))) return GROUTER_ERR_CUDA;
 
-  // compute (caller's stream)
+  // compute (caller's stream); with overlap on, dY is gathered beside the forward products and the combine runs beside the
+  // backward pass's first kernels, both on the context's side stream
   if (!ok(cudaStreamWaitEvent(st, ctx->ev_in_fwd[set], 0))) return GROUTER_ERR_CUDA;
   int rc = grouter_plan(ctx, sb + sg.idx, fold_map, reinterpret_cast<int32_t*>(sb + sg.counts), reinterpret_cast<int32_t*>(sb + sg.offsets),
                         reinterpret_cast<int32_t*>(sb + sg.r2s), reinterpret_cast<int32_t*>(sb + sg.s2r), stream);
   if (rc != GROUTER_OK) return rc;
+  const bool side = ctx->overlap && ctx->idle_gap_us == 0 && !(dm.flags & GROUTER_FLAG_FUSED_COMBINE);
+  if (side) {
+    const Workspace ws = carve_workspace(dm, ctx->R_pad_max, workspace);
+    if (!ok(cudaEventRecord(ctx->ev_plan_done, st)) || !ok(cudaStreamWaitEvent(ctx->s_side, ctx->ev_plan_done, 0)) ||
+        !ok(cudaStreamWaitEvent(ctx->s_side, ctx->ev_in_bwd[set], 0)))
+      return GROUTER_ERR_CUDA;
+    {
+      Timed tm(ctx, 6, ctx->s_side);
+      if (launch_scatter_rows(ctx, reinterpret_cast<const __nv_bfloat16*>(sb + sg.dY), ws.dYp, ctx->s_side) != cudaSuccess) return GROUTER_ERR_CUDA;
+    }
+    if (!ok(cudaEventRecord(ctx->ev_dy_gathered, ctx->s_side))) return GROUTER_ERR_CUDA;
+  }
+  ctx->step_combine_on_side = side;
   rc = grouter_moe_fwd(ctx, sb + sg.X, sb + sg.gates, W_gu, W_d, sb + sg.Y, workspace, stream);
+  ctx->step_combine_on_side = false;
   if (rc != GROUTER_OK) return rc;
-  if (!ok(cudaEventRecord(ctx->ev_fwd_done[set], st))) return GROUTER_ERR_CUDA;
+  if (!ok(cudaEventRecord(ctx->ev_fwd_done[set], side ? ctx->s_side : st))) return GROUTER_ERR_CUDA;     // Y is complete
   if (!ok(cudaStreamWaitEvent(st, ctx->ev_in_bwd[set], 0))) return GROUTER_ERR_CUDA;
+  ctx->step_dy_pregathered = side;
+  ctx->step_combine_on_side = side;      // bwd: the dX product waits for the combine before it reuses the buffer
   rc = grouter_moe_bwd(ctx, sb + sg.dY, sb + sg.X, sb + sg.gates, W_gu, W_d, sb + sg.dX, dW_gu, dW_d,
                        reinterpret_cast<float*>(sb + sg.dgates), workspace, stream);
+  ctx->step_dy_pregathered = ctx->step_combine_on_side = false;
   if (rc != GROUTER_OK) return rc;
   if (!ok(cudaEventRecord(ctx->ev_bwd_done[set], st))) return GROUTER_ERR_CUDA;
 
@@ -495,6 +558,12 @@ int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t
     launches[ctx->ev_slot[i]] += 1;
   }
   ctx->ev_used = 0;
+  return GROUTER_OK;
+}
+
+int grouter_set_overlap(grouter_ctx* ctx, int32_t on) {
+  if (!ctx) return GROUTER_ERR_INVALID_ARG;
+  ctx->overlap = on != 0;
   return GROUTER_OK;
 }
 

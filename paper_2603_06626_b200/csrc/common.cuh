@@ -104,6 +104,12 @@ struct grouter_ctx {
   int num_sms;
   // copy pipeline of grouter_moe_step_host: uploads, compute and downloads of consecutive steps overlap
   cudaStream_t s_in, s_out;          // host->device and device->host copy streams
+  cudaStream_t s_side;               // bandwidth-bound kernels that run beside a GEMM (see grouter_moe_bwd)
+  cudaEvent_t ev_fork, ev_zero_done, ev_dx_done, ev_join, ev_plan_done, ev_dy_gathered, ev_down_done, ev_combined;
+  // set by grouter_moe_step_host around its fwd / bwd calls: the step call may let work of one pass run beside the other
+  bool step_combine_on_side;         // fwd: the combine goes to s_side (its completion is ev_combined)
+  bool step_dy_pregathered;          // bwd: dY was gathered on s_side already (completion: ev_dy_gathered)
+  bool overlap;                      // run those kernels on s_side (default) or in line
   cudaEvent_t ev_in_fwd[2], ev_in_bwd[2], ev_fwd_done[2], ev_bwd_done[2], ev_out_done[2];   // per staging set
   int64_t host_steps;                // steps submitted so far; step i uses staging set i & 1
   // optional per-kernel timing (event pool)
