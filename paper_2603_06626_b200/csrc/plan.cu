@@ -26,6 +26,13 @@
 
 namespace grouter {
 
+// Programmatic dependent launch between the plan's three kernels: a kernel lets its successor's blocks be scheduled
+// early (launch_successor), and the successor does whatever needs none of the predecessor's results (clearing its
+// counters, loading the fold table) before it waits for the predecessor to finish and its writes to be visible
+// (wait_for_predecessor).  On a plain launch both are no-ops.
+__device__ __forceinline__ void launch_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ int bits_for(int n) { return n <= 1 ? 0 : 32 - __clz(n - 1); }
 
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
@@ -199,6 +206,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_count_kernel(const IdxT* __
   uint32_t* s_hist = sm_u32;                                                       // [PLAN_WARPS][E_tgt]
   uint16_t* s_fold = reinterpret_cast<uint16_t*>(sm_u32 + PLAN_WARPS * E_tgt);     // [E_src]
   const int tid = threadIdx.x, warp = tid >> 5;
+  launch_successor();
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) s_hist[i] = 0u;
   const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
   __syncthreads();
@@ -276,13 +284,13 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_place_kernel(const IdxT* __
   __shared__ int s_warp_sum[PLAN_WARPS];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  write_tile_list(pp, E_tgt, reinterpret_cast<int32_t*>(sm_raw + L.pp), reinterpret_cast<int32_t*>(sm_raw + L.po));
-
   {
     uint4* z = reinterpret_cast<uint4*>(s_cnt);
     for (int i = tid; i < E_tgt * CNT_ROW_WORDS / 4; i += PLAN_THREADS) z[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
+  wait_for_predecessor();      // everything below reads what phase 1 wrote
+  write_tile_list(pp, E_tgt, reinterpret_cast<int32_t*>(sm_raw + L.pp), reinterpret_cast<int32_t*>(sm_raw + L.po));
   // Per expert (E_tgt <= 256 = one per thread): this block's slot count, from the prefixes over blocks that phase 1
   // left; its exclusive scan over experts = the expert's first position in the staging array; the first global row.
   {
@@ -489,6 +497,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_hist_ballot_kernel(const Id
                                                                         int32_t* __restrict__ blk_hist, int32_t* __restrict__ status) {
   extern __shared__ int32_t sm[];  // PLAN_WARPS * E_tgt ints
   const int tid = threadIdx.x;
+  launch_successor();
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
   __syncthreads();
   warp_histogram(idx, fold_map, R, E_src, E_tgt, chunk, sm, status);
@@ -508,6 +517,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_permute_ballot_kernel(const
                                                                            int32_t* __restrict__ slot_to_row) {
   extern __shared__ int32_t sm[];  // PLAN_WARPS * E_tgt ints, then 2 * (E_tgt + 1) for the tile list
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  wait_for_predecessor();
   write_tile_list(pp, E_tgt, sm + PLAN_WARPS * E_tgt, sm + PLAN_WARPS * E_tgt + E_tgt + 1);
   for (int i = tid; i < PLAN_WARPS * E_tgt; i += PLAN_THREADS) sm[i] = 0;
   __syncthreads();
@@ -694,21 +704,32 @@ __device__ __forceinline__ void plan_layout(int32_t* sm, int E_tgt, const Padded
     }
     __syncthreads();
   }
+  // chunk entries: a thread per expert for the usual few chunks, the whole block for an expert cut into many
+  auto write_chunk = [&](int e, int c, int n, int base, int rem) {
+    const int i = c < rem ? s_wpos[e] + c : s_wpos[E_tgt + e] + (c - rem);
+    pp.wchunk_expert[i] = e | (n > 1 ? WCHUNK_SPLIT : 0);
+    pp.wchunk_row0[i] = s_pad[e] + (c * base + min(c, rem)) * ROW_TILE;
+    int rows = (base + (c < rem ? 1 : 0)) * ROW_TILE;
+    // the contraction runs in steps of 64 rows: when the expert's last block holds at most 64 real rows, its second
+    // half is all padding (zeros) and is left out
+    const int tail = s_cnt[e] & (ROW_TILE - 1);
+    if (c == n - 1 && tail >= 1 && tail <= ROW_TILE / 2) rows -= ROW_TILE / 2;
+    pp.wchunk_rows[i] = rows;
+  };
+  constexpr int MANY_CHUNKS = 16;
   for (int e = tid; e < E_tgt; e += nthr) {
     const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
     const int n = s_wch[e + 1] - s_wch[e];
+    if (n > MANY_CHUNKS) continue;
     const int base = blocks / n, rem = blocks - base * n;
-    for (int c = 0; c < n; ++c) {
-      const int i = c < rem ? s_wpos[e] + c : s_wpos[E_tgt + e] + (c - rem);
-      pp.wchunk_expert[i] = e | (n > 1 ? WCHUNK_SPLIT : 0);
-      pp.wchunk_row0[i] = s_pad[e] + (c * base + min(c, rem)) * ROW_TILE;
-      int rows = (base + (c < rem ? 1 : 0)) * ROW_TILE;
-      // the contraction runs in steps of 64 rows: when the expert's last block holds at most 64 real rows, its second
-      // half is all padding (zeros) and is left out
-      const int tail = s_cnt[e] & (ROW_TILE - 1);
-      if (c == n - 1 && tail >= 1 && tail <= ROW_TILE / 2) rows -= ROW_TILE / 2;
-      pp.wchunk_rows[i] = rows;
-    }
+    for (int c = 0; c < n; ++c) write_chunk(e, c, n, base, rem);
+  }
+  for (int e = 0; e < E_tgt; ++e) {
+    const int n = s_wch[e + 1] - s_wch[e];
+    if (n <= MANY_CHUNKS) continue;
+    const int blocks = (s_pad[e + 1] - s_pad[e]) / ROW_TILE;
+    const int base = blocks / n, rem = blocks - base * n;
+    for (int c = tid; c < n; c += nthr) write_chunk(e, c, n, base, rem);
   }
 }
 
@@ -719,6 +740,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_scan_kernel(int E_tgt, int 
   __shared__ int s_warp_sum[PLAN_WARPS];
   __shared__ int s_last;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  launch_successor();
+  wait_for_predecessor();
 
   // ---- this block's expert: exclusive prefix over blocks of its per-block counts, in place; the total is counts[e] ----
   {
@@ -791,6 +814,23 @@ static cudaError_t allow_smem(size_t bytes) {
   return e;
 }
 
+// Launch as a programmatic dependent of the previous kernel on the stream: its blocks may be scheduled before that
+// kernel has finished; the kernel itself waits (wait_for_predecessor) before it touches the predecessor's results.
+template <typename... Params, typename... Args>
+static cudaError_t launch_dependent(void (*kern)(Params...), int grid, int block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<Params>(args)...);
+}
+
 template <typename IdxT, int V>
 static cudaError_t launch_counted(grouter_ctx* ctx, int phase, const IdxT* idx, const int32_t* fold_map, int32_t* offsets,
                                   int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
@@ -805,7 +845,8 @@ static cudaError_t launch_counted(grouter_ctx* ctx, int phase, const IdxT* idx, 
     const size_t sm2 = (size_t)place_smem(dm.E_src, E, 16 * V, fold_map != nullptr).bytes;
     cudaError_t e = allow_smem<plan_place_kernel<IdxT, V>>(sm2);
     if (e != cudaSuccess) return e;
-    plan_place_kernel<IdxT, V><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, (int)ctx->R, dm.E_src, E, nblk, ctx->pp, offsets, row_to_slot, slot_to_row);
+    return launch_dependent(plan_place_kernel<IdxT, V>, nblk, PLAN_THREADS, sm2, st, idx, fold_map, (int)ctx->R, dm.E_src, E, nblk, ctx->pp,
+                            (const int32_t*)offsets, row_to_slot, slot_to_row);
   }
   return cudaGetLastError();
 }
@@ -818,8 +859,7 @@ static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, c
   const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
   if (phase == 1) {
     const size_t sm1 = sizeof(int32_t) * (size_t)plan_scan_smem_ints(E);
-    plan_scan_kernel<<<E, PLAN_THREADS, sm1, st>>>(E, nblk, ctx->pp, counts, offsets);
-    return cudaGetLastError();
+    return launch_dependent(plan_scan_kernel, E, PLAN_THREADS, sm1, st, E, nblk, ctx->pp, counts, offsets);
   }
   switch (ctx->geom.ipt) {
     case 16: return launch_counted<IdxT, 1>(ctx, phase, idx, fold_map, offsets, row_to_slot, slot_to_row, st);
@@ -832,8 +872,8 @@ static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, c
     plan_hist_ballot_kernel<IdxT><<<nblk, PLAN_THREADS, sm0, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp.blk_prefix, ctx->pp.status);
   } else {
     const size_t sm2 = sizeof(int32_t) * (size_t)(PLAN_WARPS * E + 2 * (E + 1));
-    plan_permute_ballot_kernel<IdxT><<<nblk, PLAN_THREADS, sm2, st>>>(idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp, offsets,
-                                                                      row_to_slot, slot_to_row);
+    return launch_dependent(plan_permute_ballot_kernel<IdxT>, nblk, PLAN_THREADS, sm2, st, idx, fold_map, R, dm.E_src, E, chunk, nblk, ctx->pp,
+                            (const int32_t*)offsets, row_to_slot, slot_to_row);
   }
   return cudaGetLastError();
 }
