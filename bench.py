@@ -758,9 +758,19 @@ def main():
     if world == 1 and not args.no_isolated:
         line["combine_ab"] = combine_ab_leg(dev, w, layer, idx, fm, gates, X, W_gu, W_d)
     if world == 1 and not args.no_plan_scale:
-        layer.close()
         torch.cuda.synchronize()
         time.sleep(3.0)     # the step loop ran at the power cap; these short kernels are timed on a GPU that has settled
+        for _ in range(5):
+            layer.plan(idx, fm)
+        pe0.record()
+        for _ in range(50):
+            layer.plan(idx, fm)
+        pe1.record()
+        torch.cuda.synchronize()
+        line["plan"]["ms_alone_settled"] = pe0.elapsed_time(pe1) / 50
+        line["plan"]["note_clocks"] = ("`ms`: 50 builds back to back right after the step loop, at the SM clock the power cap left; "
+                                       "`ms_alone_settled`: the same after three idle seconds")
+        layer.close()
         ps = plan_at_scale(dev)
         ps["frac_of_hbm"] = ps["gbs"] / peaks["hbm_gbs"]
         line["plan_scaled"] = ps
