@@ -48,6 +48,29 @@ def test_plan_ragged_sizes(T, k, E):
     _assert_equal(got, orc.plan(idx, None, E))
 
 
+@pytest.mark.parametrize("T,k,E,kind", [
+    (131203, 8, 128, "u8"),        # just above 2^20 slots: runs of 32 slots per thread, ragged last block
+    (131203, 8, 200, "fold_i32"),  # the same run length with 32-bit ids and a fold map onto 37 experts
+    (524301, 8, 128, "u8"),        # just above 2^22 slots: runs of 64 slots per thread, ragged last block
+    (600011, 7, 256, "skew"),      # 256 experts, most slots on a few of them (long runs of one expert inside a block)
+])
+def test_plan_longer_runs_per_thread_bit_exact(T, k, E, kind):
+    """The permutation kernel gives a thread 16, 32 or 64 consecutive slots depending on the problem size; the two longer
+    forms only appear above a million slots."""
+    rng = np.random.default_rng(T + E)
+    fm, E_tgt = None, E
+    if kind == "skew":
+        idx = (rng.random((T, k)) ** 6 * E).astype(np.int64)
+    else:
+        idx = rng.integers(0, E, size=(T, k))
+    if kind == "fold_i32":
+        E_tgt = 37
+        fm = rng.integers(0, E_tgt, size=E)
+    got, st = _run_plan(idx, fm, E, E_tgt, idx_i32=(kind == "fold_i32"))
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, fm, E_tgt))
+
+
 def test_plan_degenerate_and_i32():
     idx = np.full((3000, 2), 5)
     got, st = _run_plan(idx, None, 9, 9)
