@@ -251,6 +251,13 @@ int grouter_moe_bwd(grouter_ctx* ctx, const void* dY, const void* X, const void*
                     const void* W_d, void* dX, float* dW_gu, float* dW_d, float* dgates, void* workspace,
                     void* stream);
 
+/* A context is laid out for dims.T tokens; this makes its later calls (plan, fwd, bwd, the step call, the
+ * expert-parallel row calls) work on the first `tokens` of them only, 1 <= tokens <= dims.T: every [T, ...] argument is
+ * then a [tokens, ...] array and T*k becomes tokens*k.  Host call, no allocation; a new grouter_plan is needed
+ * afterwards.  For batches whose size changes from step to step, e.g. the rows an expert-parallel rank receives: one
+ * context for the largest batch serves them all.  The paper has no counterpart. */
+int grouter_set_active_tokens(grouter_ctx* ctx, int32_t tokens);
+
 /* grouter_moe_bwd runs two bandwidth-bound kernels (the zero-fill of split experts' gradients, the final reduction of
  * dX) on a stream the context owns, beside the tensor-core products they do not depend on, and joins them back into
  * `stream` before it returns: to the caller the call is ordered on `stream` as ever.  on = 0 puts them back in line

@@ -23,7 +23,7 @@ GATE_BF16, GATE_F32 = 0, 1
 EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grouter_host_staging_bytes", "grouter_plan",
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
-           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest", "grouter_set_overlap",
+           "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest", "grouter_set_overlap", "grouter_set_active_tokens",
            "grouter_ep_relabel_host", "grouter_ep_layout_host", "grouter_ep_expand_ids", "grouter_ep_dispatch_rows", "grouter_ep_combine_rows"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW", "plan_scan"]
@@ -106,6 +106,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_ep_dispatch_rows.restype = ctypes.c_int
     lib.grouter_ep_combine_rows.argtypes = [vp] * 7
     lib.grouter_ep_combine_rows.restype = ctypes.c_int
+    lib.grouter_set_active_tokens.argtypes = [vp, ctypes.c_int32]
+    lib.grouter_set_active_tokens.restype = ctypes.c_int
     lib.grouter_set_overlap.argtypes = [vp, ctypes.c_int32]
     lib.grouter_set_overlap.restype = ctypes.c_int
     lib.grouter_set_wait_limit.argtypes = [vp, ctypes.c_int64]
@@ -149,6 +151,7 @@ class GrouterLayer:
         self.device = torch.device(device)
         self.dims = GrouterDims(T, d, ffn, E_src, E_src if E_tgt is None else E_tgt, k, idx_dtype, gate_dtype, flags)
         self.T, self.d, self.ffn, self.k = T, d, ffn, k
+        self.T_active = T
         self.E_src, self.E_tgt = E_src, self.dims.E_tgt
         self.R = T * k
         with torch.cuda.device(self.device):
@@ -185,7 +188,8 @@ class GrouterLayer:
         self.counts / offsets / row_to_slot / slot_to_row."""
         _check(self.lib.grouter_plan(self.ctx, _ptr(idx), _ptr(fold_map), _ptr(self.counts), _ptr(self.offsets),
                                      _ptr(self.row_to_slot), _ptr(self.slot_to_row), _stream()), "grouter_plan")
-        return self.counts, self.offsets, self.row_to_slot, self.slot_to_row
+        n = self.T_active * self.k
+        return self.counts, self.offsets, self.row_to_slot[:n], self.slot_to_row[:n]
 
     def forward(self, X, gates, W_gu, W_d, Y=None):
         if Y is None:
@@ -199,7 +203,7 @@ class GrouterLayer:
         dX = torch.empty_like(X) if dX is None else dX
         dW_gu = torch.empty(W_gu.shape, **f32) if dW_gu is None else dW_gu
         dW_d = torch.empty(W_d.shape, **f32) if dW_d is None else dW_d
-        dgates = torch.empty((self.T, self.k), **f32) if dgates is None else dgates
+        dgates = torch.empty((self.T_active, self.k), **f32) if dgates is None else dgates
         _check(self.lib.grouter_moe_bwd(self.ctx, _ptr(dY), _ptr(X), _ptr(gates), _ptr(W_gu), _ptr(W_d), _ptr(dX), _ptr(dW_gu),
                                         _ptr(dW_d), _ptr(dgates), _ptr(self.workspace), _stream()), "grouter_moe_bwd")
         return dX, dW_gu, dW_d, dgates
@@ -247,6 +251,12 @@ class GrouterLayer:
         """out[t, :] = sum_j gate * rows[slot_to_row[t*k+j], :] and/or dgates[t, j] = <dY[t, :], rows[slot_to_row[t*k+j], :]>."""
         _check(self.lib.grouter_ep_combine_rows(self.ctx, _ptr(rows), _ptr(gates), _ptr(out), _ptr(dY), _ptr(dgates), _stream()),
                "grouter_ep_combine_rows")
+
+    def set_active_tokens(self, tokens: int) -> None:
+        """Later calls work on the first `tokens` tokens (<= the T the layer was created for): pass [tokens, ...] tensors.
+        The plan outputs are views of the first entries of self.counts / offsets / row_to_slot / slot_to_row."""
+        _check(self.lib.grouter_set_active_tokens(self.ctx, tokens), "grouter_set_active_tokens")
+        self.T_active = tokens
 
     def set_overlap(self, on: bool) -> None:
         """Bandwidth-bound kernels of the backward pass beside the GEMMs (default) or in line."""

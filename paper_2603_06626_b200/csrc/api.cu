@@ -171,6 +171,9 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
     c->max_wchunks = dims->E_tgt + (int)(c->R_pad_max / chunk) + 1;
   }
   c->geom = plan_geom(c->R, dims->E_src, dims->E_tgt);
+  c->T_act = dims->T;
+  c->R_act = c->R;
+  c->nblk_act = c->geom.nblk;
   c->planned = c->forwarded = false;
   c->ev_start = c->ev_stop = nullptr;
   c->ev_slot = nullptr;
@@ -306,7 +309,7 @@ int grouter_moe_fwd(grouter_ctx* ctx, const void* X, const void* gates, const vo
   }
   if (ctx->dims.flags & GROUTER_FLAG_FUSED_COMBINE) {
     // the down product adds every routed row into the token's fp32 row; a last pass rounds to bf16
-    const size_t n = (size_t)ctx->dims.T * ctx->dims.d;
+    const size_t n = (size_t)ctx->T_act * ctx->dims.d;
     {
       Timed tm(ctx, 5, st);
       if (cudaMemsetAsync(ws.Yacc, 0, n * sizeof(float), st) != cudaSuccess) return GROUTER_ERR_CUDA;
@@ -419,7 +422,7 @@ int grouter_moe_step_host(grouter_ctx* ctx, const void* idx_host, const void* ga
   const Staging sg = staging_layout(dm);
   const int set = (int)(ctx->host_steps & 1);
   char* sb = static_cast<char*>(workspace) + ws_bytes + (size_t)set * sg.bytes;
-  const size_t R = (size_t)dm.T * dm.k, Td = (size_t)dm.T * dm.d;
+  const size_t R = (size_t)ctx->T_act * dm.k, Td = (size_t)ctx->T_act * dm.d;     // copies move the active tokens only
   const size_t idx_b = R * (dm.idx_dtype == GROUTER_IDX_U8 ? 1 : 4), gate_b = R * (dm.gate_dtype == GROUTER_GATE_BF16 ? 2 : 4);
   auto ok = [](cudaError_t e) { return e == cudaSuccess; };
 
@@ -558,6 +561,15 @@ int grouter_timing_read(grouter_ctx* ctx, void* stream, float* total_ms, int32_t
     launches[ctx->ev_slot[i]] += 1;
   }
   ctx->ev_used = 0;
+  return GROUTER_OK;
+}
+
+int grouter_set_active_tokens(grouter_ctx* ctx, int32_t tokens) {
+  if (!ctx || tokens < 1 || tokens > ctx->dims.T) return GROUTER_ERR_INVALID_ARG;
+  ctx->T_act = tokens;
+  ctx->R_act = (int64_t)tokens * ctx->dims.k;
+  ctx->nblk_act = (int)((ctx->R_act + ctx->geom.chunk - 1) / ctx->geom.chunk);     // never more than the context was laid out for
+  ctx->planned = ctx->forwarded = false;      // the previous plan covered another number of tokens
   return GROUTER_OK;
 }
 

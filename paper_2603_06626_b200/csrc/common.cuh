@@ -93,6 +93,10 @@ struct grouter_ctx {
   grouter_dims dims;
   int device;
   int64_t R;
+  // tokens the calls work on (grouter_set_active_tokens; dims.T unless set lower), their slots, and the plan blocks they take
+  int32_t T_act;
+  int64_t R_act;
+  int nblk_act;
   int64_t R_pad_max;      // round_up(R,128) + 128*E_tgt
   int max_m_tiles;
   int max_wchunks;        // E_tgt + R_pad_max / (chunk rows) + 1

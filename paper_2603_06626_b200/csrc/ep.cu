@@ -218,7 +218,7 @@ int grouter_ep_expand_ids(const int32_t* seg_offsets, int32_t n_seg, int32_t n_l
 }
 
 static int ep_grid(const grouter_ctx* ctx) {
-  const int want = (ctx->dims.T + EP_WARPS - 1) / EP_WARPS, cap = ctx->num_sms * 8;
+  const int want = (ctx->T_act + EP_WARPS - 1) / EP_WARPS, cap = ctx->num_sms * 8;
   return want < cap ? (want < 1 ? 1 : want) : cap;
 }
 
@@ -229,7 +229,7 @@ int grouter_ep_dispatch_rows(grouter_ctx* ctx, const void* src, const void* gate
   const grouter_dims& dm = ctx->dims;
   ep_dispatch_rows_kernel<<<ep_grid(ctx), EP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(src), static_cast<__nv_bfloat16*>(rows), ctx->pp.slot_to_row, gates,
-      dm.gate_dtype == GROUTER_GATE_F32, dm.T, dm.k, dm.d);
+      dm.gate_dtype == GROUTER_GATE_F32, ctx->T_act, dm.k, dm.d);
   return cudaGetLastError() == cudaSuccess ? GROUTER_OK : GROUTER_ERR_CUDA;
 }
 
@@ -242,7 +242,7 @@ int grouter_ep_combine_rows(grouter_ctx* ctx, const void* rows, const void* gate
   const grouter_dims& dm = ctx->dims;
   ep_combine_rows_kernel<<<ep_grid(ctx), EP_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<const __nv_bfloat16*>(rows), ctx->pp.slot_to_row, gates, dm.gate_dtype == GROUTER_GATE_F32,
-      static_cast<__nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dY), dgates, dm.T, dm.k, dm.d);
+      static_cast<__nv_bfloat16*>(out), static_cast<const __nv_bfloat16*>(dY), dgates, ctx->T_act, dm.k, dm.d);
   return cudaGetLastError() == cudaSuccess ? GROUTER_OK : GROUTER_ERR_CUDA;
 }
 

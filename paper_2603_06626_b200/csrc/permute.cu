@@ -211,15 +211,15 @@ static int mover_grid(const grouter_ctx* ctx, int T) {
 
 cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  scatter_rows_kernel<SCATTER_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift,
-                                                                      ctx->pp.pad_begin, ctx->pp.pad_offsets, dm.T, dm.k, dm.d, dm.E_tgt);
+  scatter_rows_kernel<SCATTER_SEG><<<mover_grid(ctx, ctx->T_act), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift,
+                                                                      ctx->pp.pad_begin, ctx->pp.pad_offsets, ctx->T_act, dm.k, dm.d, dm.E_tgt);
   return cudaGetLastError();
 }
 
 cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* out, const float* dgate_part, int n_part,
                                float* dgates, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  reduce_rows_kernel<REDUCE_SEG><<<mover_grid(ctx, dm.T), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift, dm.T, dm.k, dm.d,
+  reduce_rows_kernel<REDUCE_SEG><<<mover_grid(ctx, ctx->T_act), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift, ctx->T_act, dm.k, dm.d,
                                                                      dm.E_tgt, dgate_part, n_part, (size_t)ctx->R_pad_max, dgates);
   return cudaGetLastError();
 }

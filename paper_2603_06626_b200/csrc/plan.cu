@@ -835,17 +835,17 @@ template <typename IdxT, int V>
 static cudaError_t launch_counted(grouter_ctx* ctx, int phase, const IdxT* idx, const int32_t* fold_map, int32_t* offsets,
                                   int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  const int E = dm.E_tgt, nblk = ctx->geom.nblk;
+  const int E = dm.E_tgt, nblk = ctx->nblk_act;
   if (phase == 0) {
     const size_t sm0 = (size_t)PLAN_WARPS * E * 4 + (fold_map ? (size_t)dm.E_src * 2 : 0);
     cudaError_t e = allow_smem<plan_count_kernel<IdxT, V>>(sm0);
     if (e != cudaSuccess) return e;
-    plan_count_kernel<IdxT, V><<<nblk, PLAN_THREADS, sm0, st>>>(idx, fold_map, (int)ctx->R, dm.E_src, E, nblk, ctx->pp.blk_prefix, ctx->pp.status);
+    plan_count_kernel<IdxT, V><<<nblk, PLAN_THREADS, sm0, st>>>(idx, fold_map, (int)ctx->R_act, dm.E_src, E, nblk, ctx->pp.blk_prefix, ctx->pp.status);
   } else {
     const size_t sm2 = (size_t)place_smem(dm.E_src, E, 16 * V, fold_map != nullptr).bytes;
     cudaError_t e = allow_smem<plan_place_kernel<IdxT, V>>(sm2);
     if (e != cudaSuccess) return e;
-    return launch_dependent(plan_place_kernel<IdxT, V>, nblk, PLAN_THREADS, sm2, st, idx, fold_map, (int)ctx->R, dm.E_src, E, nblk, ctx->pp,
+    return launch_dependent(plan_place_kernel<IdxT, V>, nblk, PLAN_THREADS, sm2, st, idx, fold_map, (int)ctx->R_act, dm.E_src, E, nblk, ctx->pp,
                             (const int32_t*)offsets, row_to_slot, slot_to_row);
   }
   return cudaGetLastError();
@@ -855,8 +855,8 @@ template <typename IdxT>
 static cudaError_t launch_plan_t(grouter_ctx* ctx, int phase, const IdxT* idx, const int32_t* fold_map, int32_t* counts,
                                  int32_t* offsets, int32_t* row_to_slot, int32_t* slot_to_row, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
-  const int R = (int)ctx->R, E = dm.E_tgt;
-  const int chunk = ctx->geom.chunk, nblk = ctx->geom.nblk;
+  const int R = (int)ctx->R_act, E = dm.E_tgt;
+  const int chunk = ctx->geom.chunk, nblk = ctx->nblk_act;
   if (phase == 1) {
     const size_t sm1 = sizeof(int32_t) * (size_t)plan_scan_smem_ints(E);
     return launch_dependent(plan_scan_kernel, E, PLAN_THREADS, sm1, st, E, nblk, ctx->pp, counts, offsets);
@@ -984,6 +984,9 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.dims.idx_dtype = idx_dtype; c.dims.gate_dtype = GROUTER_GATE_BF16;
   c.R = (int64_t)T * k;
   c.geom = plan_geom(c.R, E_src, E_tgt);
+  c.T_act = T;
+  c.R_act = c.R;
+  c.nblk_act = c.geom.nblk;
   c.pp.pad_offsets = base + NA_PAD_OFFSETS;
   c.pp.row_shift = base + NA_ROW_SHIFT;
   c.pp.pad_begin = base + NA_PAD_BEGIN;

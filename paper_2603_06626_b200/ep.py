@@ -60,7 +60,8 @@ class ExpertParallelRank:
     """One rank of the expert-parallel layer: its T tokens (source side) and its experts (expert side)."""
 
     def __init__(self, rank: int, world: int, T: int, d: int, ffn: int, E_src: int, E_tgt: int, k: int, first_expert,
-                 device: str = "cuda:0", idx_dtype: int = binding.IDX_U8, gate_dtype: int = binding.GATE_BF16):
+                 device: str = "cuda:0", idx_dtype: int = binding.IDX_U8, gate_dtype: int = binding.GATE_BF16,
+                 max_recv_rows: Optional[int] = None):
         self.rank, self.world, self.T, self.d, self.ffn, self.k = rank, world, T, d, ffn, k
         self.E_tgt = E_tgt
         self.first_expert = _i32(first_expert)
@@ -74,11 +75,37 @@ class ExpertParallelRank:
         self.fwd_back = torch.empty((self.R, d), dtype=torch.bfloat16, device=self.device)      # the forward's returned rows, kept for dgates
         self.layout = None
         self.exp = None
+        # With max_recv_rows the expert side is laid out once for that many received rows and serves every routing
+        # table that sends this rank no more (grouter_set_active_tokens per table); without it, it is rebuilt per table.
+        self.max_recv_rows = max_recv_rows
+        self.n_local = int(self.first_expert[rank + 1] - self.first_expert[rank])
+        self.exp_active = None
+        if max_recv_rows is not None:
+            self._build_expert_side(max_recv_rows)
 
     def close(self):
         self.src.close()
         if self.exp is not None:
             self.exp.close()
+
+    def _build_expert_side(self, rows: int) -> None:
+        dev = self.device
+        i8 = self.n_local <= 256
+        self.recv_rows = torch.empty((max(rows, 1), self.d), dtype=torch.bfloat16, device=dev)    # what the experts receive
+        self.recv_rows2 = torch.empty((max(rows, 1), self.d), dtype=torch.bfloat16, device=dev)   # ... in the backward pass
+        self.out_rows = torch.empty((max(rows, 1), self.d), dtype=torch.bfloat16, device=dev)     # what the experts send back
+        if rows == 0 or self.n_local == 0:
+            return
+        self.exp = binding.GrouterLayer(rows, self.d, self.ffn, self.n_local, 1, idx_dtype=binding.IDX_U8 if i8 else binding.IDX_I32,
+                                        gate_dtype=binding.GATE_BF16, device=str(dev))
+        self.exp_ids = torch.empty((rows, 1), dtype=torch.uint8 if i8 else torch.int32, device=dev)
+        self.unit_gates = torch.ones((rows, 1), dtype=torch.bfloat16, device=dev)
+        self.exp_dgates = torch.empty((rows, 1), dtype=torch.float32, device=dev)
+
+    def set_tokens(self, T: int) -> None:
+        """This rank brings T tokens (at most what it was created for) to the next routing table."""
+        self.src.set_active_tokens(T)
+        self.T = T
 
     # ---- set-up per routing table (all of it is known before the step) ----
     def plan(self, idx: torch.Tensor, fold_map: Optional[torch.Tensor]):
@@ -91,31 +118,28 @@ class ExpertParallelRank:
         self.layout = lay
         n_recv = int(lay["recv_offsets"][-1])
         self.n_recv = n_recv
-        if self.exp is not None:
-            self.exp.close()
-            self.exp = None
         dev = self.device
-        self.recv_rows = torch.empty((max(n_recv, 1), self.d), dtype=torch.bfloat16, device=dev)    # what the experts receive
-        self.recv_rows2 = torch.empty((max(n_recv, 1), self.d), dtype=torch.bfloat16, device=dev)   # ... in the backward pass
-        self.out_rows = torch.empty((max(n_recv, 1), self.d), dtype=torch.bfloat16, device=dev)     # what the experts send back
-        if n_recv == 0:
+        if self.max_recv_rows is None:
+            if self.exp is not None:
+                self.exp.close()
+                self.exp = None
+            self._build_expert_side(n_recv)
+        elif n_recv > self.max_recv_rows:
+            raise ValueError(f"{n_recv} rows arrive at rank {self.rank}, more than the {self.max_recv_rows} it was laid out for")
+        self.exp_active = self.exp if n_recv > 0 else None
+        if self.exp_active is None:
             return
         n_local = lay["n_local"]
         i8 = n_local <= 256
-        self.exp = binding.GrouterLayer(n_recv, self.d, self.ffn, n_local, 1, idx_dtype=binding.IDX_U8 if i8 else binding.IDX_I32,
-                                        gate_dtype=binding.GATE_BF16, device=str(dev))
+        self.exp.set_active_tokens(n_recv)
         seg = torch.from_numpy(lay["recv_seg_offsets"]).to(dev)
-        ids = torch.empty((n_recv, 1), dtype=torch.uint8 if i8 else torch.int32, device=dev)
         with torch.cuda.device(dev):
             rc = self.src.lib.grouter_ep_expand_ids(seg.data_ptr(), self.world * n_local, n_local, n_recv,
-                                                    binding.IDX_U8 if i8 else binding.IDX_I32, ids.data_ptr(),
+                                                    binding.IDX_U8 if i8 else binding.IDX_I32, self.exp_ids.data_ptr(),
                                                     torch.cuda.current_stream().cuda_stream)
         if rc != 0:
             raise binding.GrouterError(rc, "grouter_ep_expand_ids")
-        self.exp_ids = ids
-        self.exp.plan(ids)
-        self.unit_gates = torch.ones((n_recv, 1), dtype=torch.bfloat16, device=dev)
-        self.exp_dgates = torch.empty((n_recv, 1), dtype=torch.float32, device=dev)
+        self.exp.plan(self.exp_ids)
 
     # ---- phases ----
     def fwd_dispatch(self, X):
@@ -123,7 +147,7 @@ class ExpertParallelRank:
 
     def fwd_expert(self, W_gu_local, W_d_local):
         """Runs this rank's experts on self.recv_rows -> self.out_rows."""
-        if self.exp is not None:
+        if self.exp_active is not None:
             self.exp.forward(self.recv_rows, self.unit_gates, W_gu_local, W_d_local, self.out_rows)
         return self.out_rows
 
@@ -141,7 +165,7 @@ class ExpertParallelRank:
         f32 = dict(dtype=torch.float32, device=self.device)
         dW_gu = torch.zeros(W_gu_local.shape, **f32) if dW_gu is None else dW_gu
         dW_d = torch.zeros(W_d_local.shape, **f32) if dW_d is None else dW_d
-        if self.exp is not None:
+        if self.exp_active is not None:
             self.exp.backward(self.recv_rows2, self.recv_rows, self.unit_gates, W_gu_local, W_d_local, self.out_rows, dW_gu, dW_d,
                               self.exp_dgates)
         else:

@@ -31,31 +31,37 @@ def _exchange(ranks, src_name, dst_name, to_experts):
                 getattr(rp, dst_name)[ro:ro + n].copy_(getattr(rq, src_name)[so:so + n])
 
 
-def test_expert_parallel_step_four_emulated_ranks_matches_oracle():
+def _setup(world=4, d=128, F=192, E=12, k=3):
     from paper_2603_06626_b200 import ep
-    world, d, F, E, k = 4, 128, 192, 12, 3
-    Ts = [320, 257, 400, 96]
     owner = np.array([(5 * e + 1) % world for e in range(E)])
     owner[owner == 3] = 2                                   # rank 3 owns no expert: it only sends and receives its own rows back
     relabel, first = ep.relabel_experts(owner, world)
-    base = synth.custom_workload("ep", T=Ts[0], d=d, ffn=F, E=E, k=k, seed=77)
+    base = synth.custom_workload("ep", T=64, d=d, ffn=F, E=E, k=k, seed=77)
     W_gu_bits = np.stack([synth.expert_W_gu(base, e) for e in range(E)])
     W_d_bits = np.stack([synth.expert_W_d(base, e) for e in range(E)])
     inv = np.argsort(relabel)                               # new id -> old id
     W_gu_new, W_d_new = bits_to_bf16(W_gu_bits[inv]), bits_to_bf16(W_d_bits[inv])
+    local_w = [(W_gu_new[first[p]:first[p + 1]], W_d_new[first[p]:first[p + 1]]) for p in range(world)]
+    return owner, relabel, first, W_gu_bits, W_d_bits, local_w
+
+
+def _emulated_step_against_oracle(ranks, Ts, seed0, owner, relabel, first, W_gu_bits, W_d_bits, local_w, d=128, F=192, E=12, k=3):
+    """One routing table: plans, layouts, forward and backward through all ranks with emulated exchanges; every result
+    compared with the oracle (which works in the original expert numbering over the tokens of all ranks)."""
+    world = len(ranks)
     fold = to_dev(relabel.astype(np.int32))
-    lis, ranks = [], []
+    lis = []
     for q in range(world):
-        w = synth.custom_workload("ep", T=Ts[q], d=d, ffn=F, E=E, k=k, load="zipf", zipf_s=0.9, seed=500 + q)
+        w = synth.custom_workload("ep", T=Ts[q], d=d, ffn=F, E=E, k=k, load="zipf", zipf_s=0.9, seed=seed0 + q)
         lis.append(synth.make_layer_inputs(w, with_weights=False))
-        ranks.append(ep.ExpertParallelRank(q, world, Ts[q], d, F, E, E, k, first))
+    for r, T in zip(ranks, Ts):
+        r.set_tokens(T)                                     # a rank may be laid out for more tokens than this table brings
     counts_all = np.stack([r.plan(to_dev(li.idx), fold).cpu().numpy() for r, li in zip(ranks, lis)])
     for r in ranks:
         r.set_counts(counts_all)
         assert r.src.status() == 0
-    assert ranks[3].exp is None and sum(r.n_recv for r in ranks) == sum(Ts) * k
+    assert ranks[3].exp_active is None and sum(r.n_recv for r in ranks) == sum(Ts) * k
     dev_in = [dict(X=bits_to_bf16(li.X), dY=bits_to_bf16(li.dY), gates=bits_to_bf16(li.gates)) for li in lis]
-    local_w = [(W_gu_new[first[p]:first[p + 1]], W_d_new[first[p]:first[p + 1]]) for p in range(world)]
 
     for r, t in zip(ranks, dev_in):
         r.fwd_dispatch(t["X"])
@@ -79,7 +85,7 @@ def test_expert_parallel_step_four_emulated_ranks_matches_oracle():
     for q, li in enumerate(lis):
         Y = orc.moe_forward(f64(li.X), li.idx, f64(li.gates), weights, E)
         dX, dg = orc.moe_backward_tokens(f64(li.dY), f64(li.X), li.idx, f64(li.gates), weights, E)
-        got = dict(Y=Ys[q], dX=outs[q][0], dgates=outs[q][1])
+        got = dict(Y=Ys[q][:Ts[q]], dX=outs[q][0][:Ts[q]], dgates=outs[q][1][:Ts[q]])
         for name, want in (("Y", Y), ("dX", dX), ("dgates", dg)):
             g = got[name].double().cpu().numpy()
             assert orc.rel_frobenius(g, want) < TOL, (q, name)
@@ -92,6 +98,28 @@ def test_expert_parallel_step_four_emulated_ranks_matches_oracle():
         got_gu = dWs[p][0][relabel[e] - first[p]].double().cpu().numpy()
         got_d = dWs[p][1][relabel[e] - first[p]].double().cpu().numpy()
         assert orc.rel_frobenius(got_gu, want_gu) < TOL and orc.rel_frobenius(got_d, want_d) < TOL, e
+
+
+def test_expert_parallel_step_four_emulated_ranks_matches_oracle():
+    from paper_2603_06626_b200 import ep
+    owner, relabel, first, W_gu_bits, W_d_bits, local_w = _setup()
+    Ts = [320, 257, 400, 96]
+    ranks = [ep.ExpertParallelRank(q, 4, Ts[q], 128, 192, 12, 12, 3, first) for q in range(4)]
+    _emulated_step_against_oracle(ranks, Ts, 500, owner, relabel, first, W_gu_bits, W_d_bits, local_w)
+    assert ranks[3].exp is None
+    for r in ranks:
+        r.close()
+
+
+def test_expert_parallel_ranks_laid_out_once_serve_changing_routing_tables():
+    """The expert side is created once for the most rows a rank can receive and the source side for the most tokens; two
+    routing tables with different token counts and loads then run through the same contexts (no allocation between)."""
+    from paper_2603_06626_b200 import ep
+    owner, relabel, first, W_gu_bits, W_d_bits, local_w = _setup()
+    T_max, k = 420, 3
+    ranks = [ep.ExpertParallelRank(q, 4, T_max, 128, 192, 12, 12, k, first, max_recv_rows=4 * T_max * k) for q in range(4)]
+    _emulated_step_against_oracle(ranks, [420, 133, 256, 64], 900, owner, relabel, first, W_gu_bits, W_d_bits, local_w)
+    _emulated_step_against_oracle(ranks, [97, 420, 300, 211], 950, owner, relabel, first, W_gu_bits, W_d_bits, local_w)
     for r in ranks:
         r.close()
 

@@ -373,3 +373,34 @@ def test_issuer_cycle_accounting_counts_every_tile_and_k_step():
     for name in ("wgrad_down", "wgrad_gate_up"):
         assert got[name]["tiles"] > 0 and got[name]["k_steps"] >= got[name]["tiles"]
     layer.close()
+
+
+def test_active_tokens_on_a_larger_context_match_the_oracle():
+    """grouter_set_active_tokens: a context laid out for 1000 tokens runs a batch of 613, then one of 1000, then 77."""
+    from paper_2603_06626_b200 import binding
+    full = synth.custom_workload("act", T=1000, d=256, ffn=320, E=10, k=3, seed=31)
+    layer = binding.GrouterLayer(full.T, full.d, full.ffn, full.E_src, full.k)
+    W_gu_bits = np.stack([synth.expert_W_gu(full, e) for e in range(full.E_tgt)])
+    W_d_bits = np.stack([synth.expert_W_d(full, e) for e in range(full.E_tgt)])
+    W_gu, W_d = bits_to_bf16(W_gu_bits), bits_to_bf16(W_d_bits)
+    for n, seed in ((613, 40), (1000, 41), (77, 42)):
+        w = synth.custom_workload("act", T=n, d=full.d, ffn=full.ffn, E=full.E_src, k=full.k, load="zipf", zipf_s=1.0, seed=seed)
+        li = synth.make_layer_inputs(w, with_weights=False)
+        li.W_gu, li.W_d = W_gu_bits, W_d_bits
+        layer.set_active_tokens(n)
+        plan = [t.cpu().numpy() for t in layer.plan(to_dev(li.idx))]
+        for got, want in zip(plan, orc.plan(li.idx, None, w.E_tgt)):
+            assert np.array_equal(got, want)
+        X, dY, gates = bits_to_bf16(li.X), bits_to_bf16(li.dY), bits_to_bf16(li.gates)
+        Y = layer.forward(X, gates, W_gu, W_d)
+        dX, dW_gu, dW_d, dgates = layer.backward(dY, X, gates, W_gu, W_d)
+        layer.check_status()
+        assert Y.shape[0] == n and dgates.shape == (n, w.k)
+        out = dict(Y=Y, dX=dX, dW_gu=dW_gu, dW_d=dW_d, dgates=dgates, counts=plan[0])
+        print(n, check_full(w, li, out))
+    with pytest.raises(binding.GrouterError):
+        layer.set_active_tokens(1001)
+    layer.set_active_tokens(5)
+    with pytest.raises(binding.GrouterError):                 # a new token count needs a new plan
+        layer.forward(bits_to_bf16(li.X[:5]), bits_to_bf16(li.gates[:5]), W_gu, W_d)
+    layer.close()
