@@ -289,6 +289,21 @@ def run_expert_parallel(args, rank, local_rank, world, dev):
     ms_step = shard.max_over_ranks(e0.elapsed_time(e1), dev, world) / args.steps
     assert r.src.status() == 0 and (r.exp is None or r.exp.status() == 0)
     rows_out = int(r.layout["send_counts"].sum() - r.layout["send_counts"][rank])
+    placement = None
+    if rank == 0 and w.E_src <= 256 and w.T % 4096 == 0:
+        # What the method's sample placement (Algorithm 1) is worth on a routing table whose samples lean towards one
+        # node's experts each (synthetic stand-in; 8 nodes however many ranks this run has): rows that must cross nodes
+        # when samples are dealt out in turn against each sample on its arg-max node.
+        nodes, seq_len = 8, 4096
+        own8 = (np.arange(w.E_src) * nodes // w.E_src).astype(np.int32)
+        idx_s, _ = synth.make_idx_sample_affinity(w, seq_len, own8, nodes, boost=8.0)
+        best, _ = ep.place_samples(torch.from_numpy(idx_s).to(dev), w.E_src, seq_len, own8, nodes)
+        S = w.T // seq_len
+        placement = {"nodes": nodes, "seq_len": seq_len, "samples": S, "routed_rows": int(idx_s.size),
+                     "rows_crossing_nodes_dealt_in_turn": ep.rows_crossing_ranks(idx_s, own8, np.arange(S) % nodes, seq_len),
+                     "rows_crossing_nodes_algorithm_1": ep.rows_crossing_ranks(idx_s, own8, best, seq_len),
+                     "most_samples_on_one_node": int(np.bincount(best, minlength=nodes).max()),
+                     "routing": "synthetic: each sample's home node's experts 8x as likely"}
     if rank == 0:
         peaks, peak_src = load_peaks()
         flops_rank = 18.0 * w.d * w.ffn * float(r.n_recv)
@@ -300,7 +315,8 @@ def run_expert_parallel(args, rank, local_rank, world, dev):
                              "unit": "TFLOP/s", "frac": flops_rank / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], "traffic": None,
                              "peak_source": f"{peak_src} cuBLAS bf16, sustained; the whole step (exchanges included) of rank 0's experts"},
                 "exchange": {"rows_sent_to_other_ranks_per_direction": rows_out, "bytes_per_step": 4.0 * rows_out * w.d * 2,
-                             "transfers_per_step": 4, "split_sizes": "from the plans' counts, gathered once before the timed steps"}}
+                             "transfers_per_step": 4, "split_sizes": "from the plans' counts, gathered once before the timed steps"},
+                "placement": placement}
         print(json.dumps(line))
     r.close()
 

@@ -56,6 +56,24 @@ def exchange_layout(world: int, rank: int, first_expert, counts_all):
     return out
 
 
+def place_samples(idx: torch.Tensor, E: int, seq_len: int, expert_rank, world: int):
+    """Sample placement of Algorithm 1 for expert parallelism: every sample (run of seq_len tokens of the routing table
+    `idx`, a device tensor) goes to the rank that owns at least one kept expert of most of its tokens.
+    -> (best_rank [S] int32, local_tokens [S, world] int32), both on the host; computed by grouter_routing_stats."""
+    node = torch.from_numpy(_i32(expert_rank)).to(idx.device)
+    out = binding.routing_stats(idx, E, seq_len, node, world)
+    if out["status"] != 0:
+        raise binding.GrouterError(-6, "grouter_routing_stats device status")
+    return out["best_node"].cpu().numpy(), out["local_tokens"].cpu().numpy()
+
+
+def rows_crossing_ranks(idx: np.ndarray, expert_rank, sample_rank, seq_len: int) -> int:
+    """Routed rows whose expert lives on another rank than their token, for a given sample -> rank assignment (a
+    statistic of a routing table for reporting, host side: these are the rows an expert-parallel step must transfer)."""
+    tok_rank = np.repeat(np.asarray(sample_rank), seq_len)
+    return int((np.asarray(expert_rank)[np.asarray(idx).astype(np.int64)] != tok_rank[:, None]).sum())
+
+
 class ExpertParallelRank:
     """One rank of the expert-parallel layer: its T tokens (source side) and its experts (expert side)."""
 

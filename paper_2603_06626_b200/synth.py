@@ -132,6 +132,32 @@ def make_idx(w: Workload, T: Optional[int] = None, chunk: int = 1 << 16) -> np.n
     return out
 
 
+def make_idx_sample_affinity(w: Workload, seq_len: int, owner: np.ndarray, n_nodes: int, boost: float = 8.0):
+    """Routing table whose samples (runs of seq_len tokens) lean towards the experts of one node each: a stand-in for the
+    sequence-level routing structure the paper's sample placement exploits (its corpus statistics are not available).
+
+    Sample s has a home node h(s) (seeded, uniform); the selection probability of every expert owned by h(s) is
+    multiplied by `boost` before the k distinct experts of each token are drawn as in make_idx.
+    Returns (idx [T,k], home [S])."""
+    assert w.T % seq_len == 0
+    S = w.T // seq_len
+    p = expert_probabilities(w)
+    with np.errstate(divide="ignore"):
+        logp = np.log(p)
+    rng = _rng(w.seed, _TAG_IDX, 77)
+    home = rng.integers(0, n_nodes, size=S)
+    dtype = np.uint8 if w.E_src <= 256 else np.int32
+    out = np.empty((w.T, w.k), dtype=dtype)
+    owner = np.asarray(owner)
+    for s_ in range(S):
+        lp = logp + np.log(boost) * (owner == home[s_])
+        keys = lp[None, :] + rng.gumbel(size=(seq_len, w.E_src))
+        top = np.argpartition(-keys, w.k - 1, axis=1)[:, : w.k]
+        order = np.argsort(-np.take_along_axis(keys, top, axis=1), axis=1, kind="stable")
+        out[s_ * seq_len:(s_ + 1) * seq_len] = np.take_along_axis(top, order, axis=1).astype(dtype)
+    return out, home.astype(np.int32)
+
+
 def make_gates(w: Workload, T: Optional[int] = None) -> np.ndarray:
     """bf16 bits [T,k]: softmax over the token's k chosen logits ~ N(0,1)."""
     T = w.T if T is None else T

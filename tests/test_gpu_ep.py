@@ -147,3 +147,26 @@ def test_expert_parallel_run_step_world_one_equals_the_plain_layer():
         assert orc.rel_frobenius(dW_gu[e].double().cpu().numpy(), dWo[e][0]) < TOL
         assert orc.rel_frobenius(dW_d[e].double().cpu().numpy(), dWo[e][1]) < TOL
     r.close()
+
+
+def test_sample_placement_keeps_more_rows_on_their_own_rank():
+    """Algorithm 1 as the expert-parallel layer consumes it: on a routing table whose samples lean towards one rank's
+    experts each, placing every sample on its arg-max rank leaves fewer rows to transfer than dealing samples out in turn,
+    and it finds the rank the samples were generated to prefer."""
+    from paper_2603_06626_b200 import ep
+    from oracle import stats_oracle as so
+    world, E, k, seq_len, S = 8, 64, 4, 256, 40
+    w = synth.custom_workload("place", T=S * seq_len, d=64, ffn=64, E=E, k=k, load="zipf", zipf_s=0.5, seed=3)
+    owner = (np.arange(E) * 5 % world).astype(np.int32)                 # experts dealt out over the ranks
+    idx, home = synth.make_idx_sample_affinity(w, seq_len, owner, world, boost=8.0)
+    best, local = ep.place_samples(to_dev(idx), E, seq_len, owner, world)
+    comm = so.local_tokens(idx, owner, world, seq_len)                   # the oracle's counts and choice
+    assert np.array_equal(local, comm) and np.array_equal(best, so.place_samples(comm))
+    assert (best == home).mean() > 0.9
+    dealt = np.arange(S) % world
+    cross_alg1 = ep.rows_crossing_ranks(idx, owner, best, seq_len)
+    cross_dealt = ep.rows_crossing_ranks(idx, owner, dealt, seq_len)
+    assert cross_alg1 < 0.8 * cross_dealt
+    # brute force on the definition: no other single-sample move lowers the *local-token* count criterion
+    for s_ in range(S):
+        assert comm[s_, best[s_]] == comm[s_].max()
