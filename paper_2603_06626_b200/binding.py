@@ -49,7 +49,14 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
         return _lib
     if path is None:
         path = _build.LIB
-        _build.build(force=bool(os.environ.get("GROUTER_REBUILD")))     # returns at once when the library is newer than every source
+        try:
+            _build.build(force=bool(os.environ.get("GROUTER_REBUILD")))     # returns at once when the library is newer than every source
+        except (OSError, RuntimeError) as err:
+            # no compiler here (or the build failed): an existing library is used, loudly; without one there is nothing to fall back to
+            if not os.path.exists(path):
+                raise
+            import sys
+            sys.stderr.write(f"paper_2603_06626_b200: could not rebuild libgrouter.so ({err}); loading the existing, possibly stale, library\n")
     lib = ctypes.CDLL(path)
     vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
     lib.grouter_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(GrouterDims)]
