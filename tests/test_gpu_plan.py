@@ -110,6 +110,41 @@ def test_plan_bad_index_sets_status_without_fault():
     assert st == 0                                    # status is cleared by the previous read, and contexts are separate
 
 
+def test_plan_range_checks_of_every_form():
+    """Ids are range-checked four at a time when there is no fold map (two bounds: up to 128 ids, and above), one by one
+    otherwise; a fold target out of range is reported only when a slot uses it; the ballot form serves more than 4096
+    source ids.  Every bad slot counts as expert 0 and the rest of the plan is still exact."""
+    rng = np.random.default_rng(9)
+    for E in (100, 200):                                            # both branches of the four-at-a-time check
+        idx = rng.integers(0, E, size=(3001, 4))
+        good, st = _run_plan(idx, None, E, E)
+        assert st == 0
+        _assert_equal(good, orc.plan(idx, None, E))
+        bad = idx.copy()
+        bad[1234, 2] = E + 3                                         # in range of uint8, out of range of the experts
+        got, st = _run_plan(bad, None, E, E)
+        assert st == -6
+        fixed = bad.copy(); fixed[1234, 2] = 0
+        _assert_equal(got, orc.plan(fixed, None, E))
+    # fold table with one bad target: harmless while no slot uses that source id, reported once one does
+    idx = rng.integers(0, 30, size=(2000, 3))
+    fm = rng.integers(0, 6, size=40)
+    fm[35] = 9
+    got, st = _run_plan(idx, fm, 40, 6)
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, np.where(fm < 6, fm, 0), 6))
+    idx[77, 1] = 35
+    got, st = _run_plan(idx, fm, 40, 6)
+    assert st == -6
+    _assert_equal(got, orc.plan(idx, np.where(fm < 6, fm, 0), 6))
+    # more source ids than the fold table in shared memory holds: the ballot form
+    idx = rng.integers(0, 5000, size=(1500, 2))
+    fm = rng.integers(0, 16, size=5000)
+    got, st = _run_plan(idx, fm, 5000, 16, idx_i32=True)
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, fm, 16))
+
+
 def test_host_side_errors():
     from paper_2603_06626_b200 import binding
     with pytest.raises(binding.GrouterError) as e:
