@@ -885,22 +885,51 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   }
 }
 
-// Zero-fill of the gradients that the weight-gradient GEMMs build up from several partial sums.
+// Zero-fill of the gradients that the weight-gradient GEMMs build up from several partial sums.  Every block first
+// collects the experts in question (those whose first chunk carries the split flag) into shared memory, then the grid
+// sweeps their gradient matrices with 16-byte stores.
 __global__ void __launch_bounds__(256) zero_split_dw_kernel(const int32_t* __restrict__ n_wchunks, const int32_t* __restrict__ wchunk_expert,
                                                             const int32_t* __restrict__ wchunk_row0, const int32_t* __restrict__ pad_offsets,
                                                             float4* __restrict__ dW_gu, float4* __restrict__ dW_d, size_t gu_vec4,
                                                             size_t d_vec4) {
+  constexpr int MAX_LIST = 1024;          // more split experts than this cannot exist (E_tgt <= 1024)
+  __shared__ int s_list[MAX_LIST];
+  __shared__ int s_wcnt[8];
+  __shared__ int s_n;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) s_n = 0;
+  __syncthreads();
   const int n = *n_wchunks;
+  // ordered compaction of the split experts, in chunk-list order
+  for (int base = 0; base < n; base += 256) {
+    const int ci = base + threadIdx.x;
+    int e = -1;
+    if (ci < n) {
+      const int we = wchunk_expert[ci];
+      if ((we & WCHUNK_SPLIT) && wchunk_row0[ci] == pad_offsets[we & ~WCHUNK_SPLIT]) e = we & ~WCHUNK_SPLIT;   // once per expert: at its first chunk
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, e >= 0);
+    if (lane == 0) s_wcnt[warp] = __popc(m);
+    __syncthreads();
+    int at = s_n + __popc(m & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) at += s_wcnt[w];
+    if (e >= 0 && at < MAX_LIST) s_list[at] = e;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int add = 0;
+      for (int w = 0; w < 8; ++w) add += s_wcnt[w];
+      s_n += add;
+    }
+    __syncthreads();
+  }
+  const int n_split = min(s_n, MAX_LIST);
   const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int ci = 0; ci < n; ++ci) {
-    const int we = wchunk_expert[ci];
-    if (!(we & WCHUNK_SPLIT)) continue;
-    const int e = we & ~WCHUNK_SPLIT;
-    if (wchunk_row0[ci] != pad_offsets[e]) continue;   // once per expert: at its first chunk
-    float4* gu = dW_gu + (size_t)e * gu_vec4;
-    float4* dd = dW_d + (size_t)e * d_vec4;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < gu_vec4; i += (size_t)gridDim.x * blockDim.x) gu[i] = z;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < d_vec4; i += (size_t)gridDim.x * blockDim.x) dd[i] = z;
+  const size_t first = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+  for (int j = 0; j < n_split; ++j) {
+    float4* gu = dW_gu + (size_t)s_list[j] * gu_vec4;
+    float4* dd = dW_d + (size_t)s_list[j] * d_vec4;
+    for (size_t i = first; i < gu_vec4; i += stride) gu[i] = z;
+    for (size_t i = first; i < d_vec4; i += stride) dd[i] = z;
   }
 }
 
