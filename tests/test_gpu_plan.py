@@ -173,13 +173,13 @@ def test_kernel_timing_records_and_idle_gap():
     layer = binding.GrouterLayer(w.T, 64, 64, w.E_src, w.k)
     layer.plan(idx)
     layer.timing_enable(8)
-    layer.timing_gap(20000)                    # 20 ms after each of the two plan kernels
+    layer.timing_gap(20000)                    # 20 ms after each of the three plan kernels
     torch.cuda.synchronize()
     t0 = time.time()
     layer.plan(idx)
     rec = layer.timing_read()
     waited = time.time() - t0
-    assert rec["plan_hist"][1] == 1 and rec["plan_permute"][1] == 1 and rec["plan_hist"][0] > 0
+    assert rec["plan_hist"][1] == 1 and rec["plan_scan"][1] == 1 and rec["plan_permute"][1] == 1 and rec["plan_hist"][0] > 0
     assert rec["plan_hist"][0] < 5.0           # the idle time is not part of the kernel's own record
     assert waited >= 0.035
     layer.timing_gap(0)
