@@ -2,6 +2,8 @@
 // launch sequence of the forward and backward passes.
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 using namespace grouter;
@@ -53,12 +55,20 @@ Staging staging_layout(const grouter_dims& dm) {
   return s;
 }
 
-// Brackets one kernel launch with an event pair while timing is enabled.
+// Names of the kernel slots (grouter_timing_read's order): the NVTX range around every launch carries one of them, so a
+// timeline or an `ncu --nvtx --nvtx-include` filter can address a step of the path by name.
+const char* const kSlotName[GROUTER_NUM_KERNELS] = {"plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y",
+                                                   "gather_dY", "gemm_dH", "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX",
+                                                   "zero_split_dW", "plan_scan"};
+
+// Brackets one kernel launch with an NVTX range (a no-op unless a tool is attached) and, while timing is enabled, with
+// an event pair.
 struct Timed {
   grouter_ctx* c;
   cudaStream_t st;
   int i;
   Timed(grouter_ctx* ctx, int slot, cudaStream_t s) : c(ctx), st(s), i(-1) {
+    nvtxRangePushA(kSlotName[slot]);
     if (c->ev_cap > 0 && c->ev_used < c->ev_cap) {
       i = c->ev_used++;
       c->ev_slot[i] = slot;
@@ -66,6 +76,7 @@ struct Timed {
     }
   }
   ~Timed() {
+    nvtxRangePop();
     if (i >= 0) {
       cudaEventRecord(c->ev_stop[i], st);
       if (c->idle_gap_us > 0) launch_idle(c->idle_gap_us, st);   // the next kernel starts on a GPU that has rested
