@@ -404,3 +404,37 @@ def test_active_tokens_on_a_larger_context_match_the_oracle():
     with pytest.raises(binding.GrouterError):                 # a new token count needs a new plan
         layer.forward(bits_to_bf16(li.X[:5]), bits_to_bf16(li.gates[:5]), W_gu, W_d)
     layer.close()
+
+
+def test_kernels_beside_the_gemms_change_no_bit():
+    """The backward pass runs the dX reduction and the gradient zero-fill on a stream of the context beside the GEMMs
+    (default) or in line: the same kernels on the same data, so every output is bit-identical either way, also when the
+    two forms alternate on one context."""
+    from paper_2603_06626_b200 import binding
+    w = synth.custom_workload("side", T=2048, d=512, ffn=384, E=6, k=3, load="zipf", zipf_s=1.4, seed=17)   # the hot expert is split into chunks
+    li = synth.make_layer_inputs(w)
+    layer = binding.GrouterLayer(w.T, w.d, w.ffn, w.E_src, w.k)
+    idx, gates, X, dY = to_dev(li.idx), bits_to_bf16(li.gates), bits_to_bf16(li.X), bits_to_bf16(li.dY)
+    W_gu, W_d = bits_to_bf16(li.W_gu), bits_to_bf16(li.W_d)
+    counts = None
+    results = []
+    for on in (True, False, True):
+        layer.set_overlap(on)
+        layer.plan(idx)
+        Y = layer.forward(X, gates, W_gu, W_d)
+        dX, dW_gu, dW_d, dg = layer.backward(dY, X, gates, W_gu, W_d)
+        torch.cuda.synchronize()
+        layer.check_status()
+        counts = layer.counts.cpu().numpy()
+        results.append([t.clone() for t in (Y, dX, dg, dW_gu, dW_d)])
+    whole = torch.from_numpy(((counts + 127) // 128 * 128) <= layer.wgrad_chunk_rows()).to(X.device)   # experts contracted in one piece
+    assert (~whole).any(), "the case is meant to contain an expert that is split into chunks"
+    for other in results[1:]:
+        for a, b in zip(results[0][:3], other[:3]):
+            assert torch.equal(a, b)
+        for a, b in zip(results[0][3:], other[3:]):
+            assert torch.equal(a[whole], b[whole])
+            assert (a - b).double().norm() <= 1e-6 * a.double().norm()      # chunks of a split expert are added in no fixed order
+    out = dict(Y=results[0][0], dX=results[0][1], dgates=results[0][2], dW_gu=results[0][3], dW_d=results[0][4], counts=counts)
+    print(check_full(w, li, out))
+    layer.close()
