@@ -100,3 +100,33 @@ def test_layout_rejects_inconsistent_input():
         ep.exchange_layout(2, 2, first, counts)                         # rank outside the world
     with pytest.raises(binding.GrouterError):
         ep.exchange_layout(2, 0, [0, 3, 2], counts)                     # ranges must tile [0, E)
+
+
+def test_layout_against_brute_force_on_random_cases():
+    """Host bookkeeping against the definition written out with numpy, over random worlds, owner maps and histograms
+    (some ranks without experts, some experts without rows)."""
+    rng = np.random.default_rng(2024)
+    for _ in range(60):
+        world = int(rng.integers(1, 9))
+        E = int(rng.integers(1, 40))
+        owner = rng.integers(0, world, size=E)
+        relabel, first = ep.relabel_experts(owner, world)
+        assert sorted(relabel.tolist()) == list(range(E))
+        new_owner = np.empty(E, dtype=np.int64)
+        new_owner[relabel] = owner                                   # owner of every new id: non-decreasing
+        assert np.all(np.diff(new_owner) >= 0)
+        assert [int((new_owner == r).sum()) for r in range(world)] == np.diff(first).tolist()
+        counts = rng.integers(0, 50, size=(world, E)) * (rng.random((world, E)) < 0.7)
+        for rank in range(world):
+            lay = ep.exchange_layout(world, rank, first, counts)
+            send = [int(counts[rank, new_owner == p].sum()) for p in range(world)]
+            recv = [int(counts[q, new_owner == rank].sum()) for q in range(world)]
+            assert lay["send_counts"].tolist() == send and lay["recv_counts"].tolist() == recv
+            assert lay["send_offsets"].tolist() == np.concatenate([[0], np.cumsum(send)]).tolist()
+            assert lay["recv_offsets"].tolist() == np.concatenate([[0], np.cumsum(recv)]).tolist()
+            seg = counts[:, new_owner == rank].reshape(-1)           # (source rank, local expert), source outermost
+            assert lay["recv_seg_offsets"].tolist() == np.concatenate([[0], np.cumsum(seg)]).astype(int).tolist()
+        # what every rank sends to p is what p receives
+        lays = [ep.exchange_layout(world, r, first, counts) for r in range(world)]
+        for p in range(world):
+            assert [int(lays[q]["send_counts"][p]) for q in range(world)] == lays[p]["recv_counts"].tolist()
