@@ -13,15 +13,18 @@
 //   counted (E_tgt <= 256, fold table in shared memory): a thread owns a run of 16-64 consecutive slots, fetched with
 //     16-byte loads, and a private 16-bit counter per expert in shared memory (no atomics, no warp votes).  A scan over
 //     the threads' counters gives every thread its first rank per expert; the thread then walks its run once more,
-//     handing out ranks in slot order.  The rows go to slot_to_row directly (a thread's run is contiguous there);
-//     the inverse goes through a shared-memory staging array ordered by (expert, rank), so row_to_slot is written in
-//     contiguous runs, one per expert and block.
+//     handing out ranks in slot order.  The ranks fill a shared-memory staging array ordered by (expert, rank), so
+//     row_to_slot is written in contiguous runs, one per expert and chunk, in pieces of at most 128 entries shared out
+//     among the warps; every slot's row is parked in shared memory on the way and slot_to_row leaves as one
+//     contiguous copy.  With many chunks a block takes several in turn and fetches the next one's ids while it writes
+//     the current one out.
 //   ballot (any E_tgt up to 1024, any E_src): a warp walks its sub-chunk 32 slots at a time; lanes with equal keys are
 //     found with one vote per key bit.
 // Both are bit-reproducible: no result depends on the order in which threads or blocks run.
 //
 // The fold map is the compact form of the paper's binary folding matrix M
 // (section "Expert Folding"): e_s = fold_map[idx_s].
+#include <type_traits>
 #include "common.cuh"
 
 namespace grouter {
@@ -64,6 +67,32 @@ __device__ __forceinline__ uint32_t fold_one(uint32_t raw, const FoldView& f, in
   return t & 0xffu;
 }
 
+// Target experts of 16 slots whose 8-bit ids are in registers: v = the 16 bytes at slot s (a multiple of 16), zeros at
+// or beyond R; slots at or beyond R are not checked.
+__device__ __forceinline__ uint4 check_targets16(const uint4& v, int s, int R, const FoldView& f, int& bad) {
+  uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  if (!f.plain) {
+    const int n = min(16, max(0, R - s));
+    // without a fold map a valid id is its own target: test four bytes at once for id >= E_src (bit 7 of a byte of
+    // `over`), and take the byte-by-byte path only for a word that holds a bad id, a fold table, or the ragged end
+    const uint32_t add = (uint32_t)((f.E_src <= 128 ? 128 - f.E_src : 256 - f.E_src) * 0x01010101);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (f.table == nullptr && q * 4 + 4 <= n) {
+        const uint32_t t = ((w[q] & 0x7f7f7f7fu) + add) & 0x80808080u;     // low seven bits reach the bound
+        const uint32_t over = f.E_src <= 128 ? (t | (w[q] & 0x80808080u)) : (t & w[q]);
+        if (over == 0u) continue;
+      }
+      uint32_t o = 0u;
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        if (q * 4 + b < n) o |= fold_one((w[q] >> (8 * b)) & 0xffu, f, bad) << (8 * b);
+      w[q] = o;
+    }
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 // Target experts of the 16 slots s .. s+15 as 16 bytes (slot s+i in byte i); slots at or beyond R read as 0 and are
 // not checked.  s is a multiple of 16 and idx is 16-byte aligned, so every 16-byte load is aligned and holds at least
 // one valid id: it cannot leave the page the ids end in.
@@ -71,29 +100,8 @@ template <typename IdxT>
 __device__ __forceinline__ uint4 load_targets16(const IdxT* __restrict__ idx, int s, int R, const FoldView& f, int& bad) {
   uint32_t w[4] = {0u, 0u, 0u, 0u};
   if (sizeof(IdxT) == 1) {
-    if (s < R) {
-      const uint4 v = ld_nc_v4(reinterpret_cast<const uint8_t*>(idx) + s);
-      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-    }
-    if (!f.plain) {
-      const int n = min(16, max(0, R - s));
-      // without a fold map a valid id is its own target: test four bytes at once for id >= E_src (bit 7 of a byte of
-      // `over`), and take the byte-by-byte path only for a word that holds a bad id, a fold table, or the ragged end
-      const uint32_t add = (uint32_t)((f.E_src <= 128 ? 128 - f.E_src : 256 - f.E_src) * 0x01010101);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (f.table == nullptr && q * 4 + 4 <= n) {
-          const uint32_t t = ((w[q] & 0x7f7f7f7fu) + add) & 0x80808080u;     // low seven bits reach the bound
-          const uint32_t over = f.E_src <= 128 ? (t | (w[q] & 0x80808080u)) : (t & w[q]);
-          if (over == 0u) continue;
-        }
-        uint32_t o = 0u;
-#pragma unroll
-        for (int b = 0; b < 4; ++b)
-          if (q * 4 + b < n) o |= fold_one((w[q] >> (8 * b)) & 0xffu, f, bad) << (8 * b);
-        w[q] = o;
-      }
-    }
+    const uint4 v = s < R ? ld_nc_v4(reinterpret_cast<const uint8_t*>(idx) + s) : make_uint4(0u, 0u, 0u, 0u);
+    return check_targets16(v, s, R, f, bad);
   } else {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -136,13 +144,15 @@ __device__ __forceinline__ FoldView make_fold_view(const int32_t* __restrict__ f
 // the larger value).  No half can overflow: every value stays at or below the block's slot count (at most 16384).
 constexpr int CNT_ROW_WORDS = PLAN_THREADS / 2;     // words per expert row
 
+// (32-bit registers on both: a load zero-extends into a wider register and a store takes the low half of one, so no
+// conversion instructions surround them)
 __device__ __forceinline__ uint32_t lds_u16(uint32_t addr) {
-  uint16_t v;
-  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+  uint32_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
   return v;
 }
 __device__ __forceinline__ void sts_u16(uint32_t addr, uint32_t v) {
-  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 // Shared-memory address of this thread's counter of expert 0; the one of expert e lies e * 512 bytes further.
 __device__ __forceinline__ uint32_t my_counters(const uint32_t* s_cnt) {
@@ -240,11 +250,11 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_count_kernel(const IdxT* __
   }
 }
 
-constexpr int PLACE_BIG_RUN = 1024;   // an expert with more slots than this in one block is copied out by the whole block
+constexpr int PLACE_SEG = 128;        // positions of the staging array one warp copies out at a time
 
 // Shared-memory layout of plan_place_kernel, in bytes from the start of the dynamic block.
 struct PlaceSmem {
-  int cnt, stage, first, tot, big, fold, pp, po, bytes;
+  int cnt, stage, first, seg, fold, pp, po, bytes;
 };
 __host__ __device__ inline PlaceSmem place_smem(int E_src, int E_tgt, int ipt, bool with_fold) {
   PlaceSmem m;
@@ -253,9 +263,8 @@ __host__ __device__ inline PlaceSmem place_smem(int E_src, int E_tgt, int ipt, b
   const int cnt_bytes = E_tgt * CNT_ROW_WORDS * 4, row_bytes = ipt * PLAN_THREADS * 4;
   m.cnt = take(cnt_bytes > row_bytes ? cnt_bytes : row_bytes);   // private counters; afterwards the row of every slot of the chunk
   m.stage = take(ipt * PLAN_THREADS * 2);       // slot (as its index within the chunk) at every (expert, rank) position
-  m.first = take(E_tgt * 8);                    // per expert {first staging position, first global row of this block}
-  m.tot = take(E_tgt * 4);                      // per expert: slots in this block
-  m.big = take((E_tgt + 1) * 4);                // [0] = how many, then the experts with more than PLACE_BIG_RUN slots here
+  m.first = take(E_tgt * 4);                    // per expert: first staging position
+  m.seg = take((ipt * PLAN_THREADS / PLACE_SEG + E_tgt) * 8);   // pieces of at most PLACE_SEG positions, none across two experts
   m.fold = take(with_fold ? E_src * 2 : 0);
   m.pp = take((E_tgt + 1) * 4);
   m.po = take((E_tgt + 1) * 4);
@@ -263,176 +272,225 @@ __host__ __device__ inline PlaceSmem place_smem(int E_src, int E_tgt, int ipt, b
   return m;
 }
 
-// Phase 2, counted form.
+// Phase 2, counted form.  A block takes chunks blockIdx.x, blockIdx.x + gridDim.x, ...; the ids and the per-expert
+// prefixes of its next chunk are fetched while the current one is written out.
 template <typename IdxT, int V>
-__global__ void __launch_bounds__(PLAN_THREADS) plan_place_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
-                                                                  int R, int E_src, int E_tgt, int nblk, PaddedPlan pp,
-                                                                  const int32_t* __restrict__ offsets, int32_t* __restrict__ row_to_slot,
-                                                                  int32_t* __restrict__ slot_to_row) {
+__global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT* __restrict__ idx, const int32_t* __restrict__ fold_map,
+                                                                     int R, int E_src, int E_tgt, int nblk, PaddedPlan pp,
+                                                                     const int32_t* __restrict__ offsets, int32_t* __restrict__ row_to_slot,
+                                                                     int32_t* __restrict__ slot_to_row) {
   constexpr int IPT = 16 * V;
   constexpr int CHUNK = IPT * PLAN_THREADS;
+  constexpr bool BYTES = sizeof(IdxT) == 1;     // 8-bit ids are fetched ahead as they are; wider ones are folded as they are read
   static_assert(CHUNK <= 32768, "ranks within a block are kept in 16 bits, two to a word");
   extern __shared__ __align__(16) uint8_t sm_raw[];
   const PlaceSmem L = place_smem(E_src, E_tgt, IPT, fold_map != nullptr);
   uint32_t* s_cnt = reinterpret_cast<uint32_t*>(sm_raw + L.cnt);
   uint16_t* s_stage = reinterpret_cast<uint16_t*>(sm_raw + L.stage);
   int32_t* s_rows = reinterpret_cast<int32_t*>(sm_raw + L.cnt);     // the counters' space, once they are no longer needed
-  int2* s_first = reinterpret_cast<int2*>(sm_raw + L.first);
-  int32_t* s_tot = reinterpret_cast<int32_t*>(sm_raw + L.tot);
-  int32_t* s_big = reinterpret_cast<int32_t*>(sm_raw + L.big);
+  int32_t* s_first = reinterpret_cast<int32_t*>(sm_raw + L.first);
+  int2* s_seg = reinterpret_cast<int2*>(sm_raw + L.seg);
   uint16_t* s_fold = reinterpret_cast<uint16_t*>(sm_raw + L.fold);
-  __shared__ int s_warp_sum[PLAN_WARPS];
+  __shared__ uint32_t s_warp_sum[PLAN_WARPS];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  {
-    uint4* z = reinterpret_cast<uint4*>(s_cnt);
-    for (int i = tid; i < E_tgt * CNT_ROW_WORDS / 4; i += PLAN_THREADS) z[i] = make_uint4(0u, 0u, 0u, 0u);
-  }
-  const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
-  wait_for_predecessor();      // everything below reads what phase 1 wrote
-  write_tile_list(pp, E_tgt, reinterpret_cast<int32_t*>(sm_raw + L.pp), reinterpret_cast<int32_t*>(sm_raw + L.po));
-  // Per expert (E_tgt <= 256 = one per thread): this block's slot count, from the prefixes over blocks that phase 1
-  // left; its exclusive scan over experts = the expert's first position in the staging array; the first global row.
-  {
-    const int e = tid;
-    int cnt = 0, before = 0;
-    if (e < E_tgt) {
-      const int32_t* rowp = pp.blk_prefix + (size_t)e * nblk + blockIdx.x;
-      before = __ldcg(rowp);
-      const int next = blockIdx.x + 1 < nblk ? __ldcg(rowp + 1) : __ldg(offsets + e + 1) - __ldg(offsets + e);
-      cnt = next - before;
-    }
-    int incl = cnt;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
-    }
-    if (lane == 31) s_warp_sum[warp] = incl;
-    if (tid == 0) s_big[0] = 0;
-    __syncthreads();
-    int start = incl - cnt;
-#pragma unroll
-    for (int w = 0; w < PLAN_WARPS; ++w)
-      if (w < warp) start += s_warp_sum[w];
-    if (e < E_tgt) {
-      const int first_row = __ldg(offsets + e) + before;
-      s_first[e] = make_int2(start, first_row);
-      s_tot[e] = cnt;
-      if (cnt > PLACE_BIG_RUN) s_big[1 + atomicAdd(&s_big[0], 1)] = e;
-    }
-  }
-
-  // ---- first walk: count this thread's slots per expert ----
-  const int chunk0 = blockIdx.x * CHUNK;
-  const int s0 = chunk0 + tid * IPT;
-  const int n_mine = min(IPT, max(0, R - s0));
-  const uint32_t mine = my_counters(s_cnt);
   uint4 ev[V];
-  int bad = 0;
+  auto fetch_ids = [&](int c) {
+    if (BYTES) {
+      const int s = c * CHUNK + tid * IPT;
 #pragma unroll
-  for (int v = 0; v < V; ++v) {
-    ev[v] = load_targets16<IdxT>(idx, s0 + 16 * v, R, f, bad);
-    const uint32_t w[4] = {ev[v].x, ev[v].y, ev[v].z, ev[v].w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      uint32_t before[4];
-      const int n = n_mine - (16 * v + 4 * q);
-      if (n > 0) bump4(mine, w[q], n, before);
+      for (int v = 0; v < V; ++v)
+        ev[v] = s + 16 * v < R ? ld_nc_v4(reinterpret_cast<const uint8_t*>(idx) + s + 16 * v) : make_uint4(0u, 0u, 0u, 0u);
     }
-  }
-  if (bad) atomicOr(pp.status, STATUS_BAD_INDEX);
-  __syncthreads();
-
-  // ---- exclusive scan over the threads, one expert row per warp at a time; the result starts at the expert's first
-  // staging position, so a counter then holds the staging position of its thread's next slot of that expert ----
-  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
-    uint4* rowp = reinterpret_cast<uint4*>(s_cnt + e * CNT_ROW_WORDS) + lane;    // threads 4*lane .. +3 (low) and 128 + 4*lane .. (high)
-    const uint4 a = *rowp;
-    const uint32_t sum = a.x + a.y + a.z + a.w;
-    uint32_t incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += n;
+  };
+  // Expert tid's slots in chunk c and in the chunks before it, from the prefixes over blocks that phase 1 left.
+  int cnt_e = 0, before_e = 0, off_e = 0;
+  auto fetch_prefix = [&](int c) {
+    if (tid < E_tgt) {
+      const int32_t* rowp = pp.blk_prefix + (size_t)tid * nblk + c;
+      before_e = __ldcg(rowp);
+      cnt_e = (c + 1 < nblk ? __ldcg(rowp + 1) : __ldg(offsets + tid + 1) - off_e) - before_e;
     }
-    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
-    const uint32_t start = (uint32_t)s_first[e].x;
-    // low halves count from `start`, high halves (threads 128..255) from start + (slots of threads 0..127)
-    const uint32_t x0 = incl - sum + (start | ((start + (total & 0xffffu)) << 16));
-    const uint32_t x1 = x0 + a.x, x2 = x1 + a.y, x3 = x2 + a.z;
-    *rowp = make_uint4(x0, x1, x2, x3);
-  }
-  __syncthreads();
+  };
 
-  // ---- second walk: hand out the positions in slot order ----
+  fetch_ids(blockIdx.x);                         // in flight while the block sets itself up
+  const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
+  wait_for_predecessor();                        // everything below reads what phase 1 wrote
+  if (tid < E_tgt) off_e = __ldg(offsets + tid);
+  fetch_prefix(blockIdx.x);
+  if (blockIdx.x * PLAN_THREADS < __ldg(pp.pair_prefix + E_tgt))
+    write_tile_list(pp, E_tgt, reinterpret_cast<int32_t*>(sm_raw + L.pp), reinterpret_cast<int32_t*>(sm_raw + L.po));
+  const uint32_t mine = my_counters(s_cnt);
   const uint32_t stage_addr = (uint32_t)__cvta_generic_to_shared(s_stage);
-#pragma unroll
-  for (int v = 0; v < V; ++v) {
-    const uint32_t w[4] = {ev[v].x, ev[v].y, ev[v].z, ev[v].w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int i0 = 16 * v + 4 * q;
-      const int n = n_mine - i0;
-      if (n <= 0) continue;
-      uint32_t pos[4];
-      bump4(mine, w[q], n, pos);
-#pragma unroll
-      for (int b = 0; b < 4; ++b)
-        if (b < n) sts_u16(stage_addr + 2u * pos[b], (uint32_t)(tid * IPT + i0 + b));
-    }
-  }
-  __syncthreads();
 
-  // ---- every expert's run of this block is contiguous in the staging array and in row_to_slot: the inverse permutation
-  // goes out in runs; the row of every slot is parked in shared memory (the counters are done with) ----
-  for (int e = warp; e < E_tgt; e += PLAN_WARPS) {
-    const int n = s_tot[e];
-    if (n > PLACE_BIG_RUN) continue;
-    const int2 t = s_first[e];
-    const uint16_t* src = s_stage + t.x;
-    int32_t* dst = row_to_slot + t.y;
-    int i = lane;
-    for (; i + 96 < n; i += 128) {
-      const int a = src[i], b = src[i + 32], c = src[i + 64], d = src[i + 96];
-      dst[i] = chunk0 + a;
-      dst[i + 32] = chunk0 + b;
-      dst[i + 64] = chunk0 + c;
-      dst[i + 96] = chunk0 + d;
-      s_rows[a] = t.y + i;
-      s_rows[b] = t.y + i + 32;
-      s_rows[c] = t.y + i + 64;
-      s_rows[d] = t.y + i + 96;
+  for (int c = blockIdx.x; c < nblk; c += gridDim.x) {
+    const int chunk0 = c * CHUNK;
+    const int s0 = chunk0 + tid * IPT;
+    const int n_mine = min(IPT, max(0, R - s0));
+    {
+      uint4* z = reinterpret_cast<uint4*>(s_cnt);
+      for (int i = tid; i < E_tgt * CNT_ROW_WORDS / 4; i += PLAN_THREADS) z[i] = make_uint4(0u, 0u, 0u, 0u);
     }
-    for (; i < n; i += 32) {
-      const int a = src[i];
-      dst[i] = chunk0 + a;
-      s_rows[a] = t.y + i;
-    }
-  }
-  const int n_big = s_big[0];
-  for (int j = 0; j < n_big; ++j) {
-    const int e = s_big[1 + j];
-    const int n = s_tot[e];
-    const int2 t = s_first[e];
-    for (int i = tid; i < n; i += PLAN_THREADS) {
-      const int a = s_stage[t.x + i];
-      row_to_slot[t.y + i] = chunk0 + a;
-      s_rows[a] = t.y + i;
-    }
-  }
-  __syncthreads();
-  // ---- slot_to_row: the chunk's rows, in slot order, as one contiguous copy ----
-  {
-    const int n_here = min(CHUNK, R - chunk0);
-    int32_t* dst = slot_to_row + chunk0;     // chunk0 is a multiple of 4096: 16-byte aligned
-    for (int i = 4 * tid; i < n_here; i += 4 * PLAN_THREADS) {
-      if (i + 4 <= n_here) {
-        *reinterpret_cast<int4*>(dst + i) = *reinterpret_cast<const int4*>(s_rows + i);
-      } else {
-        for (int j = i; j < n_here; ++j) dst[j] = s_rows[j];
+    // ---- per expert (E_tgt <= 256 = one per thread): exclusive scans over the experts of the slot counts (= the
+    // expert's first position in the staging array) and of the piece counts, in one word; then the expert's pieces ----
+    int n_seg;
+    {
+      const int e = tid;
+      const uint32_t both = (uint32_t)cnt_e | ((uint32_t)((cnt_e + PLACE_SEG - 1) / PLACE_SEG) << 16);   // sums stay below 2^16 each
+      uint32_t incl = both;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t n = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += n;
+      }
+      if (lane == 31) s_warp_sum[warp] = incl;
+      __syncthreads();
+      uint32_t excl = incl - both, total = 0u;
+#pragma unroll
+      for (int w = 0; w < PLAN_WARPS; ++w) {
+        const uint32_t ws = s_warp_sum[w];
+        if (w < warp) excl += ws;
+        total += ws;
+      }
+      n_seg = (int)(total >> 16);
+      if (e < E_tgt) {
+        const int start = (int)(excl & 0xffffu), first_row = off_e + before_e;
+        s_first[e] = start;
+        int2* sg = s_seg + (excl >> 16);
+        for (int i = 0; i < cnt_e; i += PLACE_SEG) *sg++ = make_int2((start + i) | (min(PLACE_SEG, cnt_e - i) << 16), first_row + i);
       }
     }
+    __syncthreads();
+
+    // ---- first walk: count this thread's slots per expert (a chunk that lies wholly below R needs no per-slot bounds) ----
+    const bool whole = chunk0 + CHUNK <= R;
+    int bad = 0;
+    auto walk1 = [&](auto whole_chunk) {
+      constexpr bool WHOLE = decltype(whole_chunk)::value;
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        if constexpr (BYTES) ev[v] = check_targets16(ev[v], s0 + 16 * v, R, f, bad);
+        else ev[v] = load_targets16<IdxT>(idx, s0 + 16 * v, R, f, bad);
+        const uint32_t w[4] = {ev[v].x, ev[v].y, ev[v].z, ev[v].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t before[4];
+          const int n = WHOLE ? 4 : n_mine - (16 * v + 4 * q);
+          if (n > 0) bump4(mine, w[q], n, before);
+        }
+      }
+    };
+    if (whole) walk1(std::true_type{}); else walk1(std::false_type{});
+    if (bad) atomicOr(pp.status, STATUS_BAD_INDEX);
+    __syncthreads();
+
+    // ---- exclusive scan over the threads, expert row by expert row (a warp keeps several rows in flight, so that their
+    // shuffle chains overlap); the result starts at the expert's first staging position, so a counter then holds the
+    // staging position of its thread's next slot of that expert ----
+    constexpr int ROWS_AT_ONCE = 4;
+    for (int e0 = warp * ROWS_AT_ONCE; e0 < E_tgt; e0 += PLAN_WARPS * ROWS_AT_ONCE) {
+      uint4 a[ROWS_AT_ONCE];
+      uint32_t sum[ROWS_AT_ONCE], incl[ROWS_AT_ONCE];
+#pragma unroll
+      for (int j = 0; j < ROWS_AT_ONCE; ++j) {
+        // lane's words: threads 4*lane .. +3 (low halves) and 128 + 4*lane .. (high halves)
+        a[j] = e0 + j < E_tgt ? reinterpret_cast<const uint4*>(s_cnt + (e0 + j) * CNT_ROW_WORDS)[lane] : make_uint4(0u, 0u, 0u, 0u);
+        sum[j] = a[j].x + a[j].y + a[j].z + a[j].w;
+        incl[j] = sum[j];
+      }
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+        for (int j = 0; j < ROWS_AT_ONCE; ++j) {
+          const uint32_t n = __shfl_up_sync(0xffffffffu, incl[j], o);
+          if (lane >= o) incl[j] += n;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < ROWS_AT_ONCE; ++j) {
+        const uint32_t total = __shfl_sync(0xffffffffu, incl[j], 31);
+        if (e0 + j < E_tgt) {
+          const uint32_t start = (uint32_t)s_first[e0 + j];
+          // low halves count from `start`, high halves (threads 128..255) from start + (slots of threads 0..127)
+          const uint32_t x0 = incl[j] - sum[j] + (start | ((start + (total & 0xffffu)) << 16));
+          const uint32_t x1 = x0 + a[j].x, x2 = x1 + a[j].y, x3 = x2 + a[j].z;
+          reinterpret_cast<uint4*>(s_cnt + (e0 + j) * CNT_ROW_WORDS)[lane] = make_uint4(x0, x1, x2, x3);
+        }
+      }
+    }
+    __syncthreads();
+
+    // ---- second walk: hand out the positions in slot order ----
+    auto walk2 = [&](auto whole_chunk) {
+      constexpr bool WHOLE = decltype(whole_chunk)::value;
+#pragma unroll
+      for (int v = 0; v < V; ++v) {
+        const uint32_t w[4] = {ev[v].x, ev[v].y, ev[v].z, ev[v].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int i0 = 16 * v + 4 * q;
+          const int n = WHOLE ? 4 : n_mine - i0;
+          if (n <= 0) continue;
+          uint32_t pos[4];
+          bump4(mine, w[q], n, pos);
+#pragma unroll
+          for (int b = 0; b < 4; ++b)
+            if (b < n) sts_u16(stage_addr + 2u * pos[b], (uint32_t)(tid * IPT + i0 + b));
+        }
+      }
+    };
+    if (whole) walk2(std::true_type{}); else walk2(std::false_type{});
+    __syncthreads();
+
+    // ---- the next chunk's ids and prefixes set out now and arrive while this chunk is written out ----
+    if (c + (int)gridDim.x < nblk) {
+      fetch_ids(c + gridDim.x);
+      fetch_prefix(c + gridDim.x);
+    }
+
+    // ---- every expert's run of this chunk is contiguous in the staging array and in row_to_slot: the inverse
+    // permutation goes out piece by piece, a warp working on two pieces at a time (the loads of both before the stores of
+    // either); the row of every slot is parked in shared memory (the counters are done with) ----
+    {
+      auto piece_load = [&](int j, int (&a)[4], int& n, int& row0) {
+        const int2 sg = s_seg[j];
+        const uint16_t* src = s_stage + (sg.x & 0xffff);
+        n = sg.x >> 16;
+        row0 = sg.y + lane;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) a[q] = lane + 32 * q < n ? (int)src[lane + 32 * q] : 0;
+      };
+      auto piece_store = [&](const int (&a)[4], int n, int row0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (lane + 32 * q < n) {
+            row_to_slot[row0 + 32 * q] = chunk0 + a[q];
+            s_rows[a[q]] = row0 + 32 * q;
+          }
+      };
+      for (int j = warp; j < n_seg; j += 2 * PLAN_WARPS) {
+        int a0[4], a1[4], n0, n1 = 0, r0, r1 = 0;
+        piece_load(j, a0, n0, r0);
+        if (j + PLAN_WARPS < n_seg) piece_load(j + PLAN_WARPS, a1, n1, r1);
+        piece_store(a0, n0, r0);
+        piece_store(a1, n1, r1);
+      }
+    }
+    __syncthreads();
+
+    // ---- slot_to_row: the chunk's rows, in slot order, as one contiguous copy ----
+    {
+      const int n_here = min(CHUNK, R - chunk0);
+      int32_t* dst = slot_to_row + chunk0;     // chunk0 is a multiple of 4096: 16-byte aligned
+      for (int i = 4 * tid; i < n_here; i += 4 * PLAN_THREADS) {
+        if (i + 4 <= n_here) {
+          *reinterpret_cast<int4*>(dst + i) = *reinterpret_cast<const int4*>(s_rows + i);
+        } else {
+          for (int j = i; j < n_here; ++j) dst[j] = s_rows[j];
+        }
+      }
+    }
+    __syncthreads();      // the rows are read before the next chunk's counters take their place
   }
 }
 
@@ -845,7 +903,11 @@ static cudaError_t launch_counted(grouter_ctx* ctx, int phase, const IdxT* idx, 
     const size_t sm2 = (size_t)place_smem(dm.E_src, E, 16 * V, fold_map != nullptr).bytes;
     cudaError_t e = allow_smem<plan_place_kernel<IdxT, V>>(sm2);
     if (e != cudaSuccess) return e;
-    return launch_dependent(plan_place_kernel<IdxT, V>, nblk, PLAN_THREADS, sm2, st, idx, fold_map, (int)ctx->R_act, dm.E_src, E, nblk, ctx->pp,
+    // two blocks fit an SM (one with more than 128 experts); with many chunks a block takes every grid-th one.  A context
+    // that does not know the SM count (the one grouter_plan_noalloc builds: at most 128 chunks) gets a block per chunk.
+    const int resident = 2 * ctx->num_sms;
+    const int grid = ctx->num_sms > 0 && nblk > 4 * resident ? resident : nblk;   // few chunks per block would only unbalance the blocks
+    return launch_dependent(plan_place_kernel<IdxT, V>, grid, PLAN_THREADS, sm2, st, idx, fold_map, (int)ctx->R_act, dm.E_src, E, nblk, ctx->pp,
                             (const int32_t*)offsets, row_to_slot, slot_to_row);
   }
   return cudaGetLastError();
