@@ -303,20 +303,24 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
         ev[v] = s + 16 * v < R ? ld_nc_v4(reinterpret_cast<const uint8_t*>(idx) + s + 16 * v) : make_uint4(0u, 0u, 0u, 0u);
     }
   };
-  // Expert tid's slots in chunk c and in the chunks before it, from the prefixes over blocks that phase 1 left.
-  int cnt_e = 0, before_e = 0, off_e = 0;
+  // Expert tid's slots in the chunks before chunk c and up to its end, from the prefixes over blocks that phase 1 left.
+  // Nothing is computed from the two values here: the loads stay in flight until the next chunk's set-up reads them.
+  int before_e = 0, upto_e = 0, off_e = 0, total_e = 0;
   auto fetch_prefix = [&](int c) {
     if (tid < E_tgt) {
       const int32_t* rowp = pp.blk_prefix + (size_t)tid * nblk + c;
       before_e = __ldcg(rowp);
-      cnt_e = (c + 1 < nblk ? __ldcg(rowp + 1) : __ldg(offsets + tid + 1) - off_e) - before_e;
+      upto_e = c + 1 < nblk ? __ldcg(rowp + 1) : total_e;
     }
   };
 
   fetch_ids(blockIdx.x);                         // in flight while the block sets itself up
   const FoldView f = make_fold_view<IdxT>(fold_map, E_src, E_tgt, s_fold);
   wait_for_predecessor();                        // everything below reads what phase 1 wrote
-  if (tid < E_tgt) off_e = __ldg(offsets + tid);
+  if (tid < E_tgt) {
+    off_e = __ldg(offsets + tid);
+    total_e = __ldg(offsets + tid + 1) - off_e;
+  }
   fetch_prefix(blockIdx.x);
   if (blockIdx.x * PLAN_THREADS < __ldg(pp.pair_prefix + E_tgt))
     write_tile_list(pp, E_tgt, reinterpret_cast<int32_t*>(sm_raw + L.pp), reinterpret_cast<int32_t*>(sm_raw + L.po));
@@ -335,7 +339,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
     // expert's first position in the staging array) and of the piece counts, in one word; then the expert's pieces ----
     int n_seg;
     {
-      const int e = tid;
+      const int e = tid, cnt_e = upto_e - before_e;
       const uint32_t both = (uint32_t)cnt_e | ((uint32_t)((cnt_e + PLACE_SEG - 1) / PLACE_SEG) << 16);   // sums stay below 2^16 each
       uint32_t incl = both;
 #pragma unroll
@@ -449,31 +453,34 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
     }
 
     // ---- every expert's run of this chunk is contiguous in the staging array and in row_to_slot: the inverse
-    // permutation goes out piece by piece, a warp working on two pieces at a time (the loads of both before the stores of
-    // either); the row of every slot is parked in shared memory (the counters are done with) ----
-    {
-      auto piece_load = [&](int j, int (&a)[4], int& n, int& row0) {
-        const int2 sg = s_seg[j];
-        const uint16_t* src = s_stage + (sg.x & 0xffff);
-        n = sg.x >> 16;
-        row0 = sg.y + lane;
+    // permutation goes out piece by piece.  A warp takes pieces warp, warp + 8, ...: every lane fetches one piece's
+    // description, the warp then works through them four at a time, the staging loads of all four before any store
+    // (shared-memory latency is long while the SM's other block walks its counters).  The row of every slot is parked
+    // in shared memory (the counters are done with) ----
+    for (int j0 = warp; j0 < n_seg; j0 += 32 * PLAN_WARPS) {
+      const int jm = j0 + lane * PLAN_WARPS;
+      const int2 my = jm < n_seg ? s_seg[jm] : make_int2(0, 0);        // length 0: nothing to do
+      const int n_here = min(32, (n_seg - j0 + PLAN_WARPS - 1) / PLAN_WARPS);
+      for (int i = 0; i < n_here; i += 4) {
+        int a[4][4], n[4], row0[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) a[q] = lane + 32 * q < n ? (int)src[lane + 32 * q] : 0;
-      };
-      auto piece_store = [&](const int (&a)[4], int n, int row0) {
+        for (int u = 0; u < 4; ++u) {
+          const int sx = __shfl_sync(0xffffffffu, my.x, (i + u) & 31), sy = __shfl_sync(0xffffffffu, my.y, (i + u) & 31);
+          const uint16_t* src = s_stage + (sx & 0xffff);
+          n[u] = sx >> 16;
+          row0[u] = sy + lane;
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-          if (lane + 32 * q < n) {
-            row_to_slot[row0 + 32 * q] = chunk0 + a[q];
-            s_rows[a[q]] = row0 + 32 * q;
-          }
-      };
-      for (int j = warp; j < n_seg; j += 2 * PLAN_WARPS) {
-        int a0[4], a1[4], n0, n1 = 0, r0, r1 = 0;
-        piece_load(j, a0, n0, r0);
-        if (j + PLAN_WARPS < n_seg) piece_load(j + PLAN_WARPS, a1, n1, r1);
-        piece_store(a0, n0, r0);
-        piece_store(a1, n1, r1);
+          for (int q = 0; q < 4; ++q) a[u][q] = lane + 32 * q < n[u] ? (int)src[lane + 32 * q] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (lane + 32 * q < n[u]) {
+              row_to_slot[row0[u] + 32 * q] = chunk0 + a[u][q];
+              s_rows[a[u][q]] = row0[u] + 32 * q;
+            }
+        }
       }
     }
     __syncthreads();
@@ -482,11 +489,22 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
     {
       const int n_here = min(CHUNK, R - chunk0);
       int32_t* dst = slot_to_row + chunk0;     // chunk0 is a multiple of 4096: 16-byte aligned
-      for (int i = 4 * tid; i < n_here; i += 4 * PLAN_THREADS) {
-        if (i + 4 <= n_here) {
-          *reinterpret_cast<int4*>(dst + i) = *reinterpret_cast<const int4*>(s_rows + i);
-        } else {
-          for (int j = i; j < n_here; ++j) dst[j] = s_rows[j];
+      if (n_here == CHUNK) {
+#pragma unroll
+        for (int i0 = 0; i0 < CHUNK; i0 += 16 * PLAN_THREADS) {       // four 16-byte loads, then four stores
+          int4 v[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) v[u] = *reinterpret_cast<const int4*>(s_rows + i0 + 4 * (u * PLAN_THREADS + tid));
+#pragma unroll
+          for (int u = 0; u < 4; ++u) *reinterpret_cast<int4*>(dst + i0 + 4 * (u * PLAN_THREADS + tid)) = v[u];
+        }
+      } else {
+        for (int i = 4 * tid; i < n_here; i += 4 * PLAN_THREADS) {
+          if (i + 4 <= n_here) {
+            *reinterpret_cast<int4*>(dst + i) = *reinterpret_cast<const int4*>(s_rows + i);
+          } else {
+            for (int j = i; j < n_here; ++j) dst[j] = s_rows[j];
+          }
         }
       }
     }
