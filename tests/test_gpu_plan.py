@@ -10,11 +10,11 @@ from tests.gpu_util import to_dev
 pytestmark = pytest.mark.gpu
 
 
-def _run_plan(idx, fold_map, E_src, E_tgt, idx_i32=False):
+def _run_plan(idx, fold_map, E_src, E_tgt, idx_i32=False, plan_only=False):
     from paper_2603_06626_b200 import binding
     T, k = idx.shape
     idx_np = idx.astype(np.int32) if idx_i32 else idx.astype(np.uint8)
-    layer = binding.GrouterLayer(T, 64, 64, E_src, k, E_tgt=E_tgt,
+    layer = binding.GrouterLayer(T, 64, 64, E_src, k, E_tgt=E_tgt, plan_only=plan_only,
                                  idx_dtype=binding.IDX_I32 if idx_i32 else binding.IDX_U8)
     fm = None if fold_map is None else to_dev(fold_map.astype(np.int32))
     out = layer.plan(to_dev(idx_np), fm)
@@ -67,6 +67,28 @@ def test_plan_longer_runs_per_thread_bit_exact(T, k, E, kind):
         E_tgt = 37
         fm = rng.integers(0, E_tgt, size=E)
     got, st = _run_plan(idx, fm, E, E_tgt, idx_i32=(kind == "fold_i32"))
+    assert st == 0
+    _assert_equal(got, orc.plan(idx, fm, E_tgt))
+
+
+@pytest.mark.parametrize("T,k,E,kind", [
+    (2500003, 8, 128, "u8"),       # 1221 chunks of 16384 slots, ragged last one
+    (2600001, 8, 256, "skew_fold"),  # 8-bit ids folded onto 96 experts, most slots on a few of them
+])
+def test_plan_many_chunks_per_block_bit_exact(T, k, E, kind):
+    """With more than eight chunks per SM the permutation kernel's blocks stay resident and take several chunks in turn,
+    fetching the next one's ids while the current one is written out."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert -(-T * k // 16384) > 8 * sms, "the case no longer reaches the resident form on this GPU"
+    rng = np.random.default_rng(T + E)
+    fm, E_tgt = None, E
+    if kind == "skew_fold":
+        idx = (rng.random((T, k)) ** 5 * E).astype(np.int64)
+        E_tgt = 96
+        fm = rng.integers(0, E_tgt, size=E)
+    else:
+        idx = rng.integers(0, E, size=(T, k))
+    got, st = _run_plan(idx, fm, E, E_tgt, plan_only=True)
     assert st == 0
     _assert_equal(got, orc.plan(idx, fm, E_tgt))
 
