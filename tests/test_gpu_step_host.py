@@ -1,6 +1,7 @@
 """grouter_moe_step_host (host buffers in and out, copies pipelined against the compute) against the device-resident
 calls: the same kernels run on the same bits, so the results must be identical, also when consecutive steps with
-different inputs are in flight together and share the two device staging sets."""
+different inputs are in flight together and share the two device staging sets.  The last step's host results are also
+checked against the oracle, so the host path does not rest on the device path alone."""
 import numpy as np
 import pytest
 import torch
@@ -61,4 +62,12 @@ def test_step_host_matches_device_calls_with_steps_in_flight(name, n_steps):
     # is not fixed: equal up to that reordering
     for got, want in ((dW_gu.cpu(), expected[-1][3]), (dW_d.cpu(), expected[-1][4])):
         assert (got - want).double().norm() <= 1e-6 * want.double().norm()
+    # the last step against the oracle (weights drawn from `base`, the step's other inputs from its own seed)
+    from dataclasses import replace
+    from tests.test_gpu_layer import check_full
+    li = replace(steps[-1], W_gu=np.stack([synth.expert_W_gu(base, e) for e in range(base.E_tgt)]),
+                 W_d=np.stack([synth.expert_W_d(base, e) for e in range(base.E_tgt)]))
+    out = dict(Y=h["Y"].view(torch.bfloat16), dX=h["dX"].view(torch.bfloat16), dgates=h["dg"], dW_gu=dW_gu.cpu(), dW_d=dW_d.cpu(),
+               counts=np.bincount(li.idx.reshape(-1), minlength=base.E_tgt))
+    check_full(base, li, out)
     layer.close()
