@@ -50,7 +50,8 @@ enum {
   GROUTER_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed                 */
   GROUTER_ERR_BAD_INDEX = -6,     /* device saw an expert id or fold target out of range */
   GROUTER_ERR_TIMEOUT = -7,       /* a bounded device-side wait ran out                */
-  GROUTER_ERR_NO_DEVICE = -8      /* no usable CUDA device / not sm_100                */
+  GROUTER_ERR_NO_DEVICE = -8,     /* no usable CUDA device / not sm_100                */
+  GROUTER_ERR_BOUNDS = -9         /* checked build only: a kernel met an index outside its array (see grouter_checked_build) */
 };
 
 enum { GROUTER_IDX_U8 = 0, GROUTER_IDX_I32 = 1 };
@@ -307,6 +308,17 @@ int grouter_set_wait_limit(grouter_ctx* ctx, int64_t microseconds);
  * writes how long the kernel waited to *waited_microseconds (host).  grouter_status then reports
  * GROUTER_ERR_TIMEOUT once and clears it. */
 int grouter_wait_selftest(grouter_ctx* ctx, int64_t limit_microseconds, int64_t* waited_microseconds, void* stream);
+
+/* No counterpart in the paper: a development aid in place of a memory checker.  Returns 1 when the library was compiled
+ * with -DGROUTER_DEBUG_BOUNDS (paper_2603_06626_b200.build.build(debug=True) -> libgrouter_debug.so), else 0.  In that
+ * build the kernels test every index they take from data before they use it: the entries of the caller's
+ * slot_to_row / row_to_slot that the row movers and the GEMM epilogues follow, the staging positions, piece and
+ * work-list slots of the plan kernels.  A value outside its array sets a sticky status bit and the access is skipped;
+ * the kernel finishes and grouter_status() returns GROUTER_ERR_BOUNDS (after GROUTER_ERR_TIMEOUT, before
+ * GROUTER_ERR_BAD_INDEX, when several are set).  Results are the same as the release build's on valid inputs.  The
+ * release build contains none of these tests: there a corrupted permutation array is the caller's error, as any bad
+ * pointer is. */
+int grouter_checked_build(void);
 
 /* Per-kernel device timing (measurement aid; no counterpart in the paper).
  * grouter_timing_enable(ctx, n) creates n CUDA event pairs (host call, allocates;

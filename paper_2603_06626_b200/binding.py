@@ -6,6 +6,7 @@ library cannot be loaded this module raises.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 from typing import Optional
@@ -24,6 +25,7 @@ EXPORTS = ["grouter_create", "grouter_destroy", "grouter_workspace_bytes", "grou
            "grouter_moe_fwd", "grouter_moe_bwd", "grouter_moe_step_host", "grouter_status", "grouter_strerror",
            "grouter_dense_gemm", "grouter_timing_enable", "grouter_timing_read", "grouter_plan_noalloc", "grouter_host_wait", "grouter_route", "grouter_route_workspace_bytes", "grouter_routing_stats",
            "grouter_fold_greedy_host", "grouter_timing_gap", "grouter_wgrad_chunk_rows", "grouter_gemm_cycles_enable", "grouter_gemm_cycles_read", "grouter_set_wait_limit", "grouter_wait_selftest", "grouter_set_overlap", "grouter_set_active_tokens",
+           "grouter_checked_build",
            "grouter_ep_relabel_host", "grouter_ep_layout_host", "grouter_ep_expand_ids", "grouter_ep_dispatch_rows", "grouter_ep_combine_rows"]
 KERNEL_SLOTS = ["plan_hist", "plan_permute", "gather_X", "gemm_up_swiglu", "gemm_down", "combine_Y", "gather_dY", "gemm_dH",
                 "wgrad_down", "gemm_dX", "wgrad_gate_up", "reduce_dX", "zero_split_dW", "plan_scan"]
@@ -123,9 +125,27 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.grouter_wait_selftest.restype = ctypes.c_int
     lib.grouter_timing_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
     lib.grouter_timing_read.restype = ctypes.c_int
+    lib.grouter_checked_build.argtypes = []
+    lib.grouter_checked_build.restype = ctypes.c_int
     if path == _build.LIB:
         _lib = lib
     return lib
+
+
+@contextlib.contextmanager
+def checked_build():
+    """Inside the block every call of this module goes through the checked build of the library (compiled on demand):
+    kernels that test data-derived indices before use and report GROUTER_ERR_BOUNDS (-9) through the status word."""
+    global _lib
+    release = load_library()
+    lib = load_library(_build.build(debug=True))
+    if lib.grouter_checked_build() != 1:
+        raise RuntimeError("libgrouter_debug.so was not compiled with the index tests")
+    _lib = lib
+    try:
+        yield lib
+    finally:
+        _lib = release
 
 
 def strerror(code: int) -> str:

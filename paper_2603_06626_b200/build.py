@@ -1,4 +1,5 @@
-"""Builds the CUDA library in-tree: csrc/*.cu -> libgrouter.so (sm_100a only)."""
+"""Builds the CUDA library in-tree: csrc/*.cu -> libgrouter.so (sm_100a only); with debug=True the checked build
+libgrouter_debug.so, whose kernels test data-derived indices before use (grouter_checked_build in the header)."""
 from __future__ import annotations
 
 import os
@@ -9,6 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libgrouter.so")
+LIB_DEBUG = os.path.join(PKG, "libgrouter_debug.so")
 SOURCES = ["api.cu", "plan.cu", "permute.cu", "gemm.cu", "route.cu", "stats.cu", "ep.cu"]
 
 
@@ -17,14 +19,17 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
     """Compiles if the library is missing or older than any source.  Returns its path."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source_mtime():
-        return LIB
+    lib = LIB_DEBUG if debug else LIB
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_source_mtime():
+        return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = f"{LIB}.{os.getpid()}.tmp"      # several processes may build at once: each writes its own file, then renames it
+    tmp = f"{lib}.{os.getpid()}.tmp"      # several processes may build at once: each writes its own file, then renames it
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo", "-shared",
            "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp]
+    if debug:
+        cmd += ["-DGROUTER_DEBUG_BOUNDS"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
@@ -34,10 +39,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if res.returncode != 0:
         if os.path.exists(tmp):
             os.remove(tmp)
-        raise RuntimeError("nvcc failed building libgrouter.so")
-    os.replace(tmp, LIB)
-    return LIB
+        raise RuntimeError(f"nvcc failed building {os.path.basename(lib)}")
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

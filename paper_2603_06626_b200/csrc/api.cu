@@ -127,6 +127,8 @@ Workspace carve_workspace(const grouter_dims& dm, int64_t Rp, void* base) {
 
 extern "C" {
 
+int grouter_checked_build(void) { return grouter::DEBUG_BOUNDS ? 1 : 0; }
+
 const char* grouter_strerror(int code) {
   switch (code) {
     case GROUTER_OK: return "ok";
@@ -138,6 +140,7 @@ const char* grouter_strerror(int code) {
     case GROUTER_ERR_BAD_INDEX: return "expert id or fold target out of range (seen on device)";
     case GROUTER_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case GROUTER_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+    case GROUTER_ERR_BOUNDS: return "checked build: a kernel met an index outside its array and skipped the access";
     default: return "unknown error";
   }
 }
@@ -256,6 +259,8 @@ int grouter_create(grouter_ctx** out, const grouter_dims* dims) {
   c->pp.ticket = reinterpret_cast<unsigned int*>(b + o_tk);
   c->pp.tile_counter = c->pp.ticket + 4;   // same 256-byte slot
   c->pp.status = reinterpret_cast<int32_t*>(b + o_st);
+  c->pp.max_m_tiles = c->max_m_tiles;
+  c->pp.max_wchunks = c->max_wchunks;
   c->d_cycles = reinterpret_cast<unsigned long long*>(b + o_cy);
   c->d_waited = reinterpret_cast<unsigned long long*>(b + o_wt);
   *out = c;
@@ -511,6 +516,7 @@ int grouter_status(grouter_ctx* ctx, void* stream) {
       if (cudaMemsetAsync(ctx->pp.tile_counter, 0, sizeof(unsigned int), st) != cudaSuccess) return GROUTER_ERR_CUDA;
       return GROUTER_ERR_TIMEOUT;
     }
+    if (h & STATUS_BOUNDS) return GROUTER_ERR_BOUNDS;
     return GROUTER_ERR_BAD_INDEX;
   }
   return GROUTER_OK;

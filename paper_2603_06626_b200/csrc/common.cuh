@@ -12,6 +12,19 @@ namespace grouter {
 // Sticky device status bits (ORed into ctx->d_status).
 constexpr int STATUS_BAD_INDEX = 1;
 constexpr int STATUS_TIMEOUT = 2;
+constexpr int STATUS_BOUNDS = 4;      // checked build only
+
+// Checked build (compiled with -DGROUTER_DEBUG_BOUNDS, as paper_2603_06626_b200.build.build(debug=True) does): an index
+// that a kernel takes from data — a permutation entry, a staging position, a work-list slot — is tested before it is
+// used; a value outside its array sets STATUS_BOUNDS in the status word and the access is skipped, so the kernel ends
+// normally and grouter_status reports GROUTER_ERR_BOUNDS.  The release build compiles every test to `true`.
+#ifdef GROUTER_DEBUG_BOUNDS
+constexpr bool DEBUG_BOUNDS = true;
+#define GROUTER_CHECKED(cond, status_word) ((cond) ? true : (atomicOr((status_word), ::grouter::STATUS_BOUNDS), false))
+#else
+constexpr bool DEBUG_BOUNDS = false;
+#define GROUTER_CHECKED(cond, status_word) (true)
+#endif
 constexpr unsigned long long DEFAULT_WAIT_LIMIT_NS = 4000000000ull;   // bounded device-side waits give up after this long
 
 constexpr int ROW_TILE = 128;        // rows one CTA owns in a GEMM tile; expert segments are padded to it
@@ -81,6 +94,7 @@ struct PaddedPlan {
   int wgrad_chunk_blocks;       // longest weight-gradient chunk, in row tiles
   unsigned int* tile_counter;   // [1] next tile of the running grouped GEMM; zero between launches
   int32_t* status;        // [1] sticky status bits
+  int max_m_tiles, max_wchunks;   // entries the two work lists have room for
   // the caller's plan arrays of the latest grouter_plan (device pointers; valid until the caller overwrites them)
   const int32_t* offsets;      // [E_tgt+1]
   const int32_t* row_to_slot;  // [R]

@@ -59,6 +59,7 @@ struct GemmParams {
   const int32_t* wchunk_row0;  // device [chunks] first padded row
   const int32_t* wchunk_rows;  // device [chunks] rows, multiple of 64
   int32_t E, d, F, k;
+  int32_t n_slots;             // routed slots of the plan in use (tokens * k)
   int32_t accumulate;          // weight-gradient modes: add every tile into the caller's gradient
   int32_t M, N, K;             // DENSE: problem; WGRAD: per-expert output M x N
   int32_t tiles_m, tiles_n;    // output tiles per problem (tiles_m unused by row-parallel modes)
@@ -188,6 +189,7 @@ __device__ __forceinline__ Tile decode_tile(const GemmParams& p, int t, int rank
 __device__ __forceinline__ float gate_of_row(const GemmParams& p, int e, int prow) {
   if (prow >= __ldg(p.pad_begin + e)) return 0.f;
   const int slot = __ldg(p.row_to_slot + (prow - __ldg(p.row_shift + e)));
+  if (!GROUTER_CHECKED((unsigned)slot < (unsigned)p.n_slots, p.status)) return 0.f;   // the caller's array, checked build only
   if (p.gate_is_f32) return __ldg(reinterpret_cast<const float*>(p.gates) + slot);
   return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.gates)[slot]);
 }
@@ -595,7 +597,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int tok = -1;
         if (live) {
           const int prow = ti.row0 + r;
-          if (prow < __ldg(p.pad_begin + ti.e)) tok = __ldg(p.row_to_slot + (prow - __ldg(p.row_shift + ti.e))) / p.k;
+          if (prow < __ldg(p.pad_begin + ti.e)) {
+            const int slot = __ldg(p.row_to_slot + (prow - __ldg(p.row_shift + ti.e)));
+            if (GROUTER_CHECKED((unsigned)slot < (unsigned)p.n_slots, p.status)) tok = slot / p.k;
+          }
         }
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
@@ -816,6 +821,7 @@ cudaError_t launch_grouped_gemm(grouter_ctx* ctx, GemmMode mode, const Workspace
   p.d = d;
   p.F = F;
   p.k = dm.k;
+  p.n_slots = (int32_t)ctx->R_act;
   p.R_pad_max = ctx->R_pad_max;
   p.accumulate = (dm.flags & GROUTER_FLAG_ACCUMULATE_DW) ? 1 : 0;
   p.row_to_slot = ctx->pp.row_to_slot;

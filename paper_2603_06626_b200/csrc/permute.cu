@@ -49,6 +49,15 @@ __device__ __forceinline__ int padded_row(int row, const int32_t* s_off, const i
   return row + s_shift[lo];
 }
 
+// The same for a row taken from the caller's slot_to_row; the checked build returns -1 (and sets the status bit) for a
+// row outside [0, offsets[E]) or a padded row outside the buffers' rows_cap rows, and the movers skip such a slot.
+__device__ __forceinline__ int checked_padded_row(int row, const int32_t* s_off, const int32_t* s_shift, int E, int rows_cap,
+                                                  int32_t* status) {
+  if (!GROUTER_CHECKED((unsigned)row < (unsigned)s_off[E], status)) return -1;
+  const int prow = padded_row(row, s_off, s_shift, E);
+  return GROUTER_CHECKED((unsigned)prow < (unsigned)rows_cap, status) ? prow : -1;
+}
+
 // SEG: 16-byte units each lane holds per pass; a warp moves SEG * 512 contiguous bytes of a row at a time.
 template <int SEG>
 __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst,
@@ -56,7 +65,8 @@ __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_b
                                                                     const int32_t* __restrict__ offsets,
                                                                     const int32_t* __restrict__ row_shift,
                                                                     const int32_t* __restrict__ pad_begin,
-                                                                    const int32_t* __restrict__ pad_offsets, int T, int k, int d, int E) {
+                                                                    const int32_t* __restrict__ pad_offsets, int T, int k, int d, int E,
+                                                                    int rows_cap, int32_t* __restrict__ status) {
   __shared__ int32_t s_off[MAX_EXPERTS + 1], s_shift[MAX_EXPERTS];
   load_layout(offsets, row_shift, E, s_off, s_shift);
   const int lane = threadIdx.x & 31;
@@ -64,7 +74,7 @@ __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_b
   const int nwarps = gridDim.x * MOVE_WARPS;
   const int units = d >> 3;  // 16-byte units per row
   for (int t = gwarp; t < T; t += nwarps) {
-    const int my_prow = lane < k ? padded_row(__ldg(slot_to_row + (size_t)t * k + lane), s_off, s_shift, E) : 0;
+    const int my_prow = lane < k ? checked_padded_row(__ldg(slot_to_row + (size_t)t * k + lane), s_off, s_shift, E, rows_cap, status) : 0;
     const char* s = reinterpret_cast<const char*>(src + (size_t)t * d);
     for (int u0 = 0; u0 < units; u0 += 32 * SEG) {
       uint4 v[SEG];
@@ -75,6 +85,7 @@ __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_b
       }
       for (int j = 0; j < k; ++j) {
         const int prow = __shfl_sync(0xffffffffu, my_prow, j);
+        if (DEBUG_BOUNDS && prow < 0) continue;
         char* o = reinterpret_cast<char*>(dst + (size_t)prow * d);
 #pragma unroll
         for (int i = 0; i < SEG; ++i) {
@@ -88,6 +99,7 @@ __global__ void __launch_bounds__(MOVE_THREADS) scatter_rows_kernel(const __nv_b
   const uint4 z = make_uint4(0u, 0u, 0u, 0u);
   for (int e = gwarp; e < E; e += nwarps) {
     const int r0 = pad_begin[e], r1 = pad_offsets[e + 1];
+    if (!GROUTER_CHECKED(r0 >= 0 && r1 <= rows_cap && r1 - r0 < ROW_TILE, status)) continue;
     for (int r = r0; r < r1; ++r) {
       char* o = reinterpret_cast<char*>(dst + (size_t)r * d);
       for (int u = lane; u < units; u += 32) st_v4(o + (size_t)u * 16, z);
@@ -113,7 +125,7 @@ __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bf
                                                                    const int32_t* __restrict__ offsets,
                                                                    const int32_t* __restrict__ row_shift, int T, int k, int d, int E,
                                                                    const float* __restrict__ dgate_part, int n_part, size_t part_stride,
-                                                                   float* __restrict__ dgates) {
+                                                                   float* __restrict__ dgates, int32_t* __restrict__ status) {
   __shared__ int32_t s_off[MAX_EXPERTS + 1], s_shift[MAX_EXPERTS];
   load_layout(offsets, row_shift, E, s_off, s_shift);
   const int lane = threadIdx.x & 31;
@@ -121,10 +133,10 @@ __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bf
   const int nwarps = gridDim.x * MOVE_WARPS;
   const int units = d >> 3;
   for (int t = gwarp; t < T; t += nwarps) {
-    const int my_prow = lane < k ? padded_row(__ldg(slot_to_row + (size_t)t * k + lane), s_off, s_shift, E) : 0;
+    const int my_prow = lane < k ? checked_padded_row(__ldg(slot_to_row + (size_t)t * k + lane), s_off, s_shift, E, (int)part_stride, status) : 0;
     if (dgates != nullptr && lane < k) {
       float g = 0.f;
-      for (int n = 0; n < n_part; ++n) g += dgate_part[(size_t)n * part_stride + my_prow];
+      for (int n = 0; n < n_part && (!DEBUG_BOUNDS || my_prow >= 0); ++n) g += dgate_part[(size_t)n * part_stride + my_prow];
       dgates[(size_t)t * k + lane] = g;
     }
     char* o = reinterpret_cast<char*>(out + (size_t)t * d);
@@ -136,6 +148,7 @@ __global__ void __launch_bounds__(MOVE_THREADS) reduce_rows_kernel(const __nv_bf
         for (int c = 0; c < 8; ++c) acc[i][c] = 0.f;
       for (int j = 0; j < k; ++j) {          // slot order: the sum is deterministic
         const int prow = __shfl_sync(0xffffffffu, my_prow, j);
+        if (DEBUG_BOUNDS && prow < 0) continue;
         const char* s = reinterpret_cast<const char*>(src + (size_t)prow * d);
         uint4 v[SEG];
 #pragma unroll
@@ -212,7 +225,7 @@ static int mover_grid(const grouter_ctx* ctx, int T) {
 cudaError_t launch_scatter_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_bfloat16* dst, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
   scatter_rows_kernel<SCATTER_SEG><<<mover_grid(ctx, ctx->T_act), MOVE_THREADS, 0, st>>>(src, dst, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift,
-                                                                      ctx->pp.pad_begin, ctx->pp.pad_offsets, ctx->T_act, dm.k, dm.d, dm.E_tgt);
+                                                                      ctx->pp.pad_begin, ctx->pp.pad_offsets, ctx->T_act, dm.k, dm.d, dm.E_tgt, (int)ctx->R_pad_max, ctx->pp.status);
   return cudaGetLastError();
 }
 
@@ -220,7 +233,7 @@ cudaError_t launch_reduce_rows(grouter_ctx* ctx, const __nv_bfloat16* src, __nv_
                                float* dgates, cudaStream_t st) {
   const grouter_dims& dm = ctx->dims;
   reduce_rows_kernel<REDUCE_SEG><<<mover_grid(ctx, ctx->T_act), MOVE_THREADS, 0, st>>>(src, out, ctx->pp.slot_to_row, ctx->pp.offsets, ctx->pp.row_shift, ctx->T_act, dm.k, dm.d,
-                                                                     dm.E_tgt, dgate_part, n_part, (size_t)ctx->R_pad_max, dgates);
+                                                                     dm.E_tgt, dgate_part, n_part, (size_t)ctx->R_pad_max, dgates, ctx->pp.status);
   return cudaGetLastError();
 }
 

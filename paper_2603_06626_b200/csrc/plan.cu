@@ -197,6 +197,7 @@ __device__ __forceinline__ void write_tile_list(const PaddedPlan& pp, int E_tgt,
       if (s_pp[mid] <= t) lo = mid; else hi = mid;
     }
     const int row0 = s_po[lo] + (t - s_pp[lo]) * 2 * ROW_TILE;
+    if (!GROUTER_CHECKED(t < pp.max_m_tiles, pp.status)) continue;
     pp.pair_row0[t] = row0;
     pp.pair_expert[t] = lo | (row0 + ROW_TILE < s_po[lo + 1] ? PAIR_VALID2 : 0);
   }
@@ -357,11 +358,14 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
         total += ws;
       }
       n_seg = (int)(total >> 16);
+      if (!GROUTER_CHECKED(n_seg <= CHUNK / PLACE_SEG + E_tgt, pp.status)) n_seg = 0;
       if (e < E_tgt) {
         const int start = (int)(excl & 0xffffu), first_row = off_e + before_e;
         s_first[e] = start;
         int2* sg = s_seg + (excl >> 16);
-        for (int i = 0; i < cnt_e; i += PLACE_SEG) *sg++ = make_int2((start + i) | (min(PLACE_SEG, cnt_e - i) << 16), first_row + i);
+        const bool fits = GROUTER_CHECKED(cnt_e >= 0 && start + cnt_e <= CHUNK && (int)(excl >> 16) + (cnt_e + PLACE_SEG - 1) / PLACE_SEG <= CHUNK / PLACE_SEG + E_tgt,
+                                          pp.status);
+        for (int i = 0; fits && i < cnt_e; i += PLACE_SEG) *sg++ = make_int2((start + i) | (min(PLACE_SEG, cnt_e - i) << 16), first_row + i);
       }
     }
     __syncthreads();
@@ -439,7 +443,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
           bump4(mine, w[q], n, pos);
 #pragma unroll
           for (int b = 0; b < 4; ++b)
-            if (b < n) sts_u16(stage_addr + 2u * pos[b], (uint32_t)(tid * IPT + i0 + b));
+            if (b < n && GROUTER_CHECKED(pos[b] < (uint32_t)CHUNK, pp.status)) sts_u16(stage_addr + 2u * pos[b], (uint32_t)(tid * IPT + i0 + b));
         }
       }
     };
@@ -468,6 +472,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
           const int sx = __shfl_sync(0xffffffffu, my.x, (i + u) & 31), sy = __shfl_sync(0xffffffffu, my.y, (i + u) & 31);
           const uint16_t* src = s_stage + (sx & 0xffff);
           n[u] = sx >> 16;
+          if (!GROUTER_CHECKED(n[u] <= PLACE_SEG && (sx & 0xffff) + n[u] <= CHUNK && sy >= 0 && sy <= R - n[u], pp.status)) n[u] = 0;
           row0[u] = sy + lane;
 #pragma unroll
           for (int q = 0; q < 4; ++q) a[u][q] = lane + 32 * q < n[u] ? (int)src[lane + 32 * q] : 0;
@@ -476,7 +481,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, 2) plan_place_kernel(const IdxT*
         for (int u = 0; u < 4; ++u) {
 #pragma unroll
           for (int q = 0; q < 4; ++q)
-            if (lane + 32 * q < n[u]) {
+            if (lane + 32 * q < n[u] && GROUTER_CHECKED(a[u][q] < CHUNK, pp.status)) {
               row_to_slot[row0[u] + 32 * q] = chunk0 + a[u][q];
               s_rows[a[u][q]] = row0[u] + 32 * q;
             }
@@ -783,6 +788,7 @@ __device__ __forceinline__ void plan_layout(int32_t* sm, int E_tgt, const Padded
   // chunk entries: a thread per expert for the usual few chunks, the whole block for an expert cut into many
   auto write_chunk = [&](int e, int c, int n, int base, int rem) {
     const int i = c < rem ? s_wpos[e] + c : s_wpos[E_tgt + e] + (c - rem);
+    if (!GROUTER_CHECKED((unsigned)i < (unsigned)pp.max_wchunks, pp.status)) return;
     pp.wchunk_expert[i] = e | (n > 1 ? WCHUNK_SPLIT : 0);
     pp.wchunk_row0[i] = s_pad[e] + (c * base + min(c, rem)) * ROW_TILE;
     int rows = (base + (c < rem ? 1 : 0)) * ROW_TILE;
@@ -1083,6 +1089,8 @@ extern "C" int grouter_plan_noalloc(const void* idx, int32_t idx_dtype, const in
   c.pp.wchunk_rows = base + NA_WCHUNK_ROWS;
   c.pp.n_wchunks = base + NA_N_WCHUNKS;
   c.pp.blk_prefix = base + NA_BLK_PREFIX;
+  c.pp.max_m_tiles = NOALLOC_MAX_ROWS / ROW_TILE;
+  c.pp.max_wchunks = NOALLOC_MAX_WCHUNKS;
   if (c.geom.nblk > NOALLOC_MAX_BLOCKS) return GROUTER_ERR_UNSUPPORTED;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
