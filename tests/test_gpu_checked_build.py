@@ -15,8 +15,10 @@ pytestmark = pytest.mark.gpu
 ERR_BOUNDS = -9
 
 
-def test_release_build_carries_no_index_tests():
+def test_release_build_carries_no_index_tests(request):
     from paper_2603_06626_b200 import binding
+    if request.config.getoption("--checked-build"):
+        pytest.skip("the session runs on the checked build")
     assert binding.load_library().grouter_checked_build() == 0
     with binding.checked_build() as lib:
         assert lib.grouter_checked_build() == 1
