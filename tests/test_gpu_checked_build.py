@@ -43,6 +43,20 @@ def test_checked_build_matches_the_oracle_and_reports_nothing(case):
     check_full(w, li, out)
 
 
+def test_both_builds_give_the_same_bits(request):
+    """No expert of this workload is split into chunks, so nothing depends on the order of atomic adds."""
+    from paper_2603_06626_b200 import binding
+    if request.config.getoption("--checked-build"):
+        pytest.skip("the session runs on the checked build")
+    w = synth.custom_workload("chk", T=1100, d=320, ffn=264, E=20, k=4, load="zipf", zipf_s=1.2, n_dead=3, seed=33)
+    li = synth.make_layer_inputs(w)
+    release = run_gpu(w, li)
+    with binding.checked_build():
+        checked = run_gpu(w, li)
+    for name in ("Y", "dX", "dgates", "dW_gu", "dW_d"):
+        assert torch.equal(release[name], checked[name]), name
+
+
 @pytest.mark.parametrize("T,k,E", [(131203, 8, 128), (40000, 6, 200)])
 def test_checked_plan_bit_exact(T, k, E):
     from paper_2603_06626_b200 import binding
